@@ -1,0 +1,143 @@
+"""TEST INFRASTRUCTURE ONLY: the CPU fp64 oracle for shared-prefix decode attention.
+
+``attend`` is a ctypes front for ``psa_oracle.c`` (the plain softmax(QK^T)V
+definition of the paper's "attn" benchmark group, two passes, fp64).
+``recurrences`` holds the paper's streaming forms of the same operator, used to
+pin the definition.  Nothing in the product imports this package; only the
+tests, the smoke check and the CPU-baseline leg of the benchmark do.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "psa_oracle.c"
+_LIB = _HERE / "libpsa_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the C oracle with gcc (OpenMP threads). Returns the library path."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", str(tmp), str(_SRC), "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [
+        ("num_prefixes", ctypes.c_int),
+        ("prefix_lens", ctypes.c_void_p),
+        ("n_samples", ctypes.c_void_p),
+        ("num_q_heads", ctypes.c_int),
+        ("num_kv_heads", ctypes.c_int),
+        ("head_dim", ctypes.c_int),
+        ("page_size", ctypes.c_int),
+        ("sm_scale", ctypes.c_double),
+        ("q", ctypes.c_void_p),
+        ("prefix_k", ctypes.c_void_p),
+        ("prefix_v", ctypes.c_void_p),
+        ("prefix_stride_tok", ctypes.c_int64),
+        ("prefix_stride_head", ctypes.c_int64),
+        ("pool_k", ctypes.c_void_p),
+        ("pool_v", ctypes.c_void_p),
+        ("pool_stride_page", ctypes.c_int64),
+        ("pool_stride_head", ctypes.c_int64),
+        ("pool_stride_tok", ctypes.c_int64),
+        ("page_indptr", ctypes.c_void_p),
+        ("page_indices", ctypes.c_void_p),
+        ("suffix_lens", ctypes.c_void_p),
+    ]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(str(build()))
+        _lib.psa_oracle_attend.restype = ctypes.c_int
+        _lib.psa_oracle_attend.argtypes = [
+            ctypes.POINTER(_Problem), ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+        ]
+        _lib.psa_oracle_weights.restype = ctypes.c_int64
+        _lib.psa_oracle_weights.argtypes = [
+            ctypes.POINTER(_Problem), ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
+        ]
+    return _lib
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _problem(w: dict):
+    """Marshal a workload dict (see the input generators) into the C struct.
+
+    Returned list keeps the numpy arrays alive for the duration of the call.
+    """
+    keep = {}
+    for name, dt in (("prefix_lens", np.int32), ("n_samples", np.int32), ("suffix_lens", np.int32),
+                     ("page_indptr", np.int32), ("page_indices", np.int32)):
+        keep[name] = _c(w[name], dt)
+    for name in ("q", "prefix_k", "prefix_v", "pool_k", "pool_v"):
+        a = w[name]
+        assert a.dtype == np.uint16, f"{name} must hold bf16 bit patterns (uint16)"
+        keep[name] = np.ascontiguousarray(a)
+    Hq, Hkv, D = int(w["num_q_heads"]), int(w["num_kv_heads"]), int(w["head_dim"])
+    page = int(w["page_size"])
+    # default layouts: prefix [sum L, Hkv, D]; pool [pages, Hkv, page, D]
+    pst = w.get("prefix_strides", (Hkv * D, D))
+    qst = w.get("pool_strides", (Hkv * page * D, page * D, D))
+    pb = _Problem(
+        len(keep["prefix_lens"]), keep["prefix_lens"].ctypes.data, keep["n_samples"].ctypes.data,
+        Hq, Hkv, D, page, float(w["sm_scale"]),
+        keep["q"].ctypes.data, keep["prefix_k"].ctypes.data, keep["prefix_v"].ctypes.data,
+        int(pst[0]), int(pst[1]),
+        keep["pool_k"].ctypes.data, keep["pool_v"].ctypes.data, int(qst[0]), int(qst[1]), int(qst[2]),
+        keep["page_indptr"].ctypes.data, keep["page_indices"].ctypes.data, keep["suffix_lens"].ctypes.data,
+    )
+    return pb, keep
+
+
+def attend(w: dict, rows=None, n_threads: int = 0):
+    """fp64 attention of every (sample, query head) row, or of ``rows`` (flat s*Hq+h).
+
+    Returns (out [n_rows, D] float64, lse [n_rows] float64, threads_used).
+    """
+    lib = _load()
+    pb, keep = _problem(w)
+    B = int(np.sum(keep["n_samples"]))
+    if rows is None:
+        n_rows, rows_ptr = B * pb.num_q_heads, None
+    else:
+        rows = _c(rows, np.int64)
+        n_rows, rows_ptr = len(rows), rows.ctypes.data
+    out = np.zeros((n_rows, pb.head_dim), dtype=np.float64)
+    lse = np.zeros((n_rows,), dtype=np.float64)
+    used = ctypes.c_int(0)
+    rc = lib.psa_oracle_attend(ctypes.byref(pb), rows_ptr, n_rows, out.ctypes.data, lse.ctypes.data,
+                               int(n_threads), ctypes.byref(used))
+    if rc != 0:
+        raise RuntimeError("psa_oracle_attend failed (bad row index or out of memory)")
+    return out, lse, used.value
+
+
+def weights(w: dict, s: int, h: int):
+    """Softmax weights of row (s, h) over its prefix-then-suffix context, fp64."""
+    lib = _load()
+    pb, keep = _problem(w)
+    cap = int(np.max(keep["prefix_lens"], initial=0)) + int(np.max(keep["suffix_lens"], initial=0)) + 1
+    buf = np.zeros((cap,), dtype=np.float64)
+    n = lib.psa_oracle_weights(ctypes.byref(pb), int(s), int(h), buf.ctypes.data, cap)
+    if n < 0:
+        raise RuntimeError("psa_oracle_weights failed")
+    return buf[:n].copy()

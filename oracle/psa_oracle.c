@@ -1,0 +1,192 @@
+/*
+ * TEST INFRASTRUCTURE ONLY -- the CPU oracle for shared-prefix decode attention.
+ *
+ * This file is the plain definition of the operator, written out in fp64 so a
+ * reader can check it by eye.  It is slow on purpose, shares nothing with the
+ * CUDA library, and may only be used by the tests, the smoke check and the
+ * CPU-baseline leg of the benchmark.  The product never calls it.
+ *
+ * Operator (paper, Appendix "Benchmark details", group "attn":
+ * softmax(S) . V with S = Q K^T; the same statement appears as the PyTorch
+ * reference of attn task 0, a softmax over the key axis followed by a batched
+ * product with V).  One decode step: every sample s of prompt p owns one query
+ * per query head h and attends, without any mask, to the L_p prompt tokens it
+ * shares with its sibling samples followed by its own S_s generated tokens.
+ * Query head h reads KV head floor(h / G), G = H_q / H_kv.
+ *
+ *   x_j   = sm_scale * sum_d q[s,h,d] * k_j[d]
+ *   m     = max_j x_j
+ *   w_j   = exp(x_j - m),  Z = sum_j w_j
+ *   out   = (sum_j w_j v_j) / Z
+ *   lse   = m + ln Z                       (natural logarithm)
+ *   empty context: out = 0, lse = -inf
+ *
+ * q, k and v arrive as bf16 bit patterns and are widened exactly.
+ * Suffix token t of sample s lives in physical page
+ * page_indices[page_indptr[s] + t / page_size], slot t % page_size.
+ *
+ * Every function here is pinned by tests/test_oracle_pins.py against closed
+ * forms, brute force, a library softmax and the paper's streaming recurrences.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_f64(uint16_t bits)
+{
+    uint32_t w = ((uint32_t)bits) << 16; /* bf16 is the top half of an IEEE float */
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+typedef struct {
+    int num_prefixes;
+    const int32_t *prefix_lens;   /* [P] */
+    const int32_t *n_samples;     /* [P] */
+    int num_q_heads, num_kv_heads, head_dim, page_size;
+    double sm_scale;
+    const uint16_t *q;            /* [B, Hq, D] */
+    const uint16_t *prefix_k, *prefix_v; /* token t of prompt p, head kv at (off_p + t)*stride_tok + kv*stride_head */
+    int64_t prefix_stride_tok, prefix_stride_head;
+    const uint16_t *pool_k, *pool_v;     /* page*stride_page + kv*stride_head + slot*stride_tok */
+    int64_t pool_stride_page, pool_stride_head, pool_stride_tok;
+    const int32_t *page_indptr;   /* [B+1] */
+    const int32_t *page_indices;
+    const int32_t *suffix_lens;   /* [B] */
+} psa_oracle_problem;
+
+/* One (sample, query head) row, two passes over the concatenated context.
+ * weights (optional, length n) receives w_j / Z. Returns the context length. */
+static int64_t attend_row(const psa_oracle_problem *pb, int prompt, int64_t prompt_tok_off,
+                          int s, int h, double *x /* scratch, >= n */,
+                          double *out, double *lse, double *weights)
+{
+    const int D = pb->head_dim;
+    const int G = pb->num_q_heads / pb->num_kv_heads;
+    const int kv = h / G;
+    const int64_t L = pb->prefix_lens[prompt];
+    const int64_t S = pb->suffix_lens[s];
+    const int64_t n = L + S;
+    const uint16_t *qrow = pb->q + ((int64_t)s * pb->num_q_heads + h) * D;
+
+    for (int d = 0; d < D; ++d) out[d] = 0.0;
+    if (n == 0) { *lse = -INFINITY; return 0; }
+
+    /* pass 1: logits and their maximum */
+    double m = -INFINITY;
+    for (int64_t j = 0; j < n; ++j) {
+        const uint16_t *krow;
+        if (j < L) {
+            krow = pb->prefix_k + (prompt_tok_off + j) * pb->prefix_stride_tok + kv * pb->prefix_stride_head;
+        } else {
+            int64_t t = j - L;
+            int64_t page = pb->page_indices[pb->page_indptr[s] + t / pb->page_size];
+            krow = pb->pool_k + page * pb->pool_stride_page + kv * pb->pool_stride_head
+                 + (t % pb->page_size) * pb->pool_stride_tok;
+        }
+        double dot = 0.0;
+        for (int d = 0; d < D; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+        x[j] = pb->sm_scale * dot;
+        if (x[j] > m) m = x[j];
+    }
+    /* pass 2: weights, normaliser, weighted sum of values */
+    double Z = 0.0;
+    for (int64_t j = 0; j < n; ++j) {
+        const uint16_t *vrow;
+        if (j < L) {
+            vrow = pb->prefix_v + (prompt_tok_off + j) * pb->prefix_stride_tok + kv * pb->prefix_stride_head;
+        } else {
+            int64_t t = j - L;
+            int64_t page = pb->page_indices[pb->page_indptr[s] + t / pb->page_size];
+            vrow = pb->pool_v + page * pb->pool_stride_page + kv * pb->pool_stride_head
+                 + (t % pb->page_size) * pb->pool_stride_tok;
+        }
+        double w = exp(x[j] - m);
+        x[j] = w;
+        Z += w;
+        for (int d = 0; d < D; ++d) out[d] += w * bf16_to_f64(vrow[d]);
+    }
+    for (int d = 0; d < D; ++d) out[d] /= Z;
+    if (weights) for (int64_t j = 0; j < n; ++j) weights[j] = x[j] / Z;
+    *lse = m + log(Z);
+    return n;
+}
+
+/* Locate the prompt a sample belongs to: samples of prompt 0 first, then prompt 1, ... */
+static void locate_sample(const psa_oracle_problem *pb, int s, int *prompt, int64_t *tok_off)
+{
+    int64_t first = 0, off = 0;
+    for (int p = 0; p < pb->num_prefixes; ++p) {
+        if (s < first + pb->n_samples[p]) { *prompt = p; *tok_off = off; return; }
+        first += pb->n_samples[p];
+        off += pb->prefix_lens[p];
+    }
+    *prompt = -1; *tok_off = 0;
+}
+
+/*
+ * Attend for a list of rows.  rows[i] = s * Hq + h selects (sample, query head);
+ * rows == NULL means all B*Hq rows in order.  out is [n_rows, D] fp64, lse [n_rows].
+ * n_threads <= 0 uses every core OpenMP sees.  Returns 0, or -1 on a bad row /
+ * allocation failure.  *threads_used (optional) reports the team size.
+ */
+int psa_oracle_attend(const psa_oracle_problem *pb, const int64_t *rows, int64_t n_rows,
+                      double *out, double *lse, int n_threads, int *threads_used)
+{
+    int64_t B = 0, max_ctx = 1;
+    for (int p = 0; p < pb->num_prefixes; ++p) B += pb->n_samples[p];
+    {
+        int64_t maxL = 0, maxS = 0;
+        for (int p = 0; p < pb->num_prefixes; ++p) if (pb->prefix_lens[p] > maxL) maxL = pb->prefix_lens[p];
+        for (int64_t s = 0; s < B; ++s) if (pb->suffix_lens[s] > maxS) maxS = pb->suffix_lens[s];
+        max_ctx = maxL + maxS + 1;
+    }
+    if (rows == NULL) n_rows = B * pb->num_q_heads;
+    int failed = 0, team = 1;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#pragma omp parallel
+#endif
+    {
+        double *x = (double *)malloc(sizeof(double) * (size_t)max_ctx);
+#ifdef _OPENMP
+#pragma omp single
+        team = omp_get_num_threads();
+#pragma omp for schedule(dynamic, 1)
+#endif
+        for (int64_t i = 0; i < n_rows; ++i) {
+            int64_t r = rows ? rows[i] : i;
+            if (!x || r < 0 || r >= B * pb->num_q_heads) { failed = 1; continue; }
+            int s = (int)(r / pb->num_q_heads), h = (int)(r % pb->num_q_heads);
+            int prompt; int64_t tok_off;
+            locate_sample(pb, s, &prompt, &tok_off);
+            if (prompt < 0) { failed = 1; continue; }
+            attend_row(pb, prompt, tok_off, s, h, x, out + i * pb->head_dim, lse + i, NULL);
+        }
+        free(x);
+    }
+    if (threads_used) *threads_used = team;
+    return failed ? -1 : 0;
+}
+
+/* Softmax weights w_j / Z of one row over its concatenated context (length L_p + S_s). */
+int64_t psa_oracle_weights(const psa_oracle_problem *pb, int s, int h, double *weights, int64_t capacity)
+{
+    int prompt; int64_t tok_off;
+    locate_sample(pb, s, &prompt, &tok_off);
+    if (prompt < 0) return -1;
+    int64_t n = (int64_t)pb->prefix_lens[prompt] + pb->suffix_lens[s];
+    if (n > capacity) return -1;
+    double *x = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    double *o = (double *)malloc(sizeof(double) * (size_t)pb->head_dim);
+    double l;
+    if (!x || !o) { free(x); free(o); return -1; }
+    attend_row(pb, prompt, tok_off, s, h, x, o, &l, weights);
+    free(x); free(o);
+    return n;
+}

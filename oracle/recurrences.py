@@ -1,0 +1,124 @@
+"""TEST INFRASTRUCTURE ONLY: the paper's streaming forms of softmax(S).V, in fp64.
+
+The paper prints three algebraically equal ways to fold a stream of
+(logit, value) pairs into the attention output (figure "attn tasks": Task 0
+normalises at every step, Task 1 splits the running maximum from the running
+sum, Task 2 defers the division to the end).  They are restated here from the
+mathematics, one scalar step at a time, so the tests can tie the two-pass
+definition in ``psa_oracle.c`` to the paper's own operator.  ``merge_partials``
+is the identity that the deferred-division form implies for contexts processed
+in pieces.  Pure Python loops: small inputs only.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) exactly: bf16 is the top half of an fp32."""
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def gather_context(w: dict, s: int, h: int):
+    """Dense fp64 copies of one row's query, keys and values (prefix first, then the
+    sample's own paged tokens), found by walking the page table here in Python."""
+    Hq, Hkv, D, page = (int(w[k]) for k in ("num_q_heads", "num_kv_heads", "head_dim", "page_size"))
+    G = Hq // Hkv
+    kv = h // G
+    n_samples = np.asarray(w["n_samples"])
+    prefix_lens = np.asarray(w["prefix_lens"])
+    first = np.concatenate([[0], np.cumsum(n_samples)])
+    p = int(np.searchsorted(first, s, side="right") - 1)
+    tok_off = int(np.sum(prefix_lens[:p]))
+    L, S = int(prefix_lens[p]), int(w["suffix_lens"][s])
+    q = bf16_bits_to_f64(np.asarray(w["q"]).reshape(-1, Hq, D)[s, h])
+    pk = np.asarray(w["prefix_k"]).reshape(-1, Hkv, D)
+    pv = np.asarray(w["prefix_v"]).reshape(-1, Hkv, D)
+    K = [pk[tok_off + t, kv] for t in range(L)]
+    V = [pv[tok_off + t, kv] for t in range(L)]
+    poolk = np.asarray(w["pool_k"]).reshape(-1, Hkv, page, D)
+    poolv = np.asarray(w["pool_v"]).reshape(-1, Hkv, page, D)
+    for t in range(S):
+        pg = int(w["page_indices"][int(w["page_indptr"][s]) + t // page])
+        K.append(poolk[pg, kv, t % page])
+        V.append(poolv[pg, kv, t % page])
+    if L + S == 0:
+        return q, np.zeros((0, D)), np.zeros((0, D))
+    return q, bf16_bits_to_f64(np.stack(K)), bf16_bits_to_f64(np.stack(V))
+
+
+def logits(w: dict, s: int, h: int):
+    """(x [n], V [n, D]) with x_j = sm_scale * q.k_j, fp64."""
+    q, K, V = gather_context(w, s, h)
+    return float(w["sm_scale"]) * (K @ q), V
+
+
+def task0_maxsum(x, V):
+    """Task 0 ("MaxSum"): running max m, running sum l, output normalised at every step.
+    State starts at (-inf, 0, 0)."""
+    D = V.shape[1]
+    m, l, o = -math.inf, 0.0, np.zeros(D)
+    for s_t, v_t in zip(x, V):
+        m_next = max(m, s_t)
+        l_prime = math.exp(m - m_next) * l
+        p = math.exp(s_t - m_next)
+        l_next = p + l_prime
+        o = (l_prime * o + p * v_t) / l_next
+        m, l = m_next, l_next
+    return o, m, l
+
+
+def _exp_max_diff(x):
+    """Shared first stage of Tasks 1 and 2: per step emit e = exp(s - m_new) and the
+    decay d = exp(m_old - m_new) of everything accumulated so far."""
+    m = -math.inf
+    for s_t in x:
+        m_next = max(m, s_t)
+        yield math.exp(s_t - m_next), math.exp(m - m_next), m_next
+        m = m_next
+
+
+def task1_divsum(x, V):
+    """Task 1: "ExpMaxDiff" feeds "DivSum", which keeps (l, o) with o normalised each step."""
+    D = V.shape[1]
+    l, o, m = 0.0, np.zeros(D), -math.inf
+    for (e, d, m), v_t in zip(_exp_max_diff(x), V):
+        l_prime = d * l
+        l_next = e + l_prime
+        o = (l_prime * o + e * v_t) / l_next
+        l = l_next
+    return o, m, l
+
+
+def task2_deferred(x, V):
+    """Task 2: "ExpMaxDiff" feeds two weighted sums (scalar r, vector acc) that are only
+    divided at the end -- the form every GPU attention kernel uses."""
+    D = V.shape[1]
+    r, acc, m = 0.0, np.zeros(D), -math.inf
+    for (e, d, m), v_t in zip(_exp_max_diff(x), V):
+        r = r * d + e
+        acc = acc * d + e * v_t
+    return acc / r, m, r
+
+
+def merge_partials(outs, lses):
+    """Combine normalised partial results of disjoint key sets.
+
+    Partial i carries out_i = sum_j w_j v_j / Z_i and lse_i = ln sum_j exp(x_j).  Since
+    the un-normalised accumulators of Task 2 simply add once brought to a common maximum,
+    lse = ln sum_i exp(lse_i) and out = sum_i exp(lse_i - lse) out_i.  Pieces with
+    lse_i = -inf are empty and contribute nothing; all empty gives (0, -inf)."""
+    lses = [float(v) for v in lses]
+    top = max(lses, default=-math.inf)
+    D = len(outs[0]) if outs else 0
+    if top == -math.inf:
+        return np.zeros(D), -math.inf
+    z = sum(math.exp(v - top) for v in lses)
+    lse = top + math.log(z)
+    out = np.zeros(D)
+    for o, v in zip(outs, lses):
+        if v != -math.inf:
+            out += math.exp(v - lse) * np.asarray(o, dtype=np.float64)
+    return out, lse
