@@ -1,0 +1,192 @@
+/*
+ * psa -- parallel-sample shared-prefix decode attention for NVIDIA B200 (sm_100a).
+ *
+ * One decode step of attention for B samples that were all drawn from the same few
+ * prompts: the paper's learning loop samples N candidate answers per task from ONE
+ * prompt made of selected demonstrations plus the task (Algorithm 1, the sampling
+ * step; appendix "Experiment details": 64 samples per temperature, at most 1024
+ * output tokens).  Every sample s of prompt p owns one query vector per query head and
+ * attends, unmasked, to the L_p prompt tokens it shares with its siblings followed by
+ * its own S_s generated tokens:
+ *
+ *     out[s,h,:] = softmax_j( sm_scale * q[s,h,:] . k_j ) . v_j ,   lse = ln sum_j exp(...)
+ *
+ * which is the operator of the paper's "attn" benchmark group, softmax(S).V with
+ * S = QK^T (appendix "Benchmark details").  The library evaluates it in three device
+ * stages and one host stage:
+ *
+ *   plan    (host)   cut prefix and suffix work into pieces that fill every SM
+ *   prefix  (device) all samples x heads of a KV head batched against the shared prefix
+ *                    K/V, read once; deferred-division online softmax (the paper's
+ *                    attn Task 2 recurrence) on tensor cores
+ *   suffix  (device) per-sample attention over ragged, paged K/V
+ *   merge   (device) log-sum-exp combination of every row's partial results
+ *
+ * Conventions
+ *   - "host" / "device" after a pointer says where the memory lives.  Every buffer is
+ *     caller-owned.  The library owns only the opaque plan (host memory).
+ *   - bf16 means the upper 16 bits of an IEEE-754 binary32, stored as uint16_t.
+ *   - Query head h reads KV head h / G, G = num_q_heads / num_kv_heads.
+ *   - Samples of prompt 0 come first in q/out/lse, then prompt 1, ...; prompts are packed
+ *     back to back along the token axis of prefix_k / prefix_v.
+ *   - No function throws, aborts or traps.  Host-detectable problems come back as a
+ *     status code; device-side problems (a bounded wait that ran out) are written to a
+ *     status word in the workspace, the affected outputs are left unwritten, and
+ *     psa_check_status reports them.
+ *   - Supported: head_dim in {64, 128}; G in {1, 2, 4, 8}; page_size 16; sm_scale > 0.
+ *     Anything else is PSA_ERR_UNSUPPORTED.  There is no fallback path of any kind.
+ */
+#ifndef PSA_H_
+#define PSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct psa_plan psa_plan_t;
+
+typedef enum {
+    PSA_OK = 0,
+    PSA_ERR_INVALID_ARG = 1, /* null pointer, negative length, misaligned buffer, ... */
+    PSA_ERR_UNSUPPORTED = 2, /* shape or dtype outside the supported set */
+    PSA_ERR_WORKSPACE = 3,   /* workspace missing, too small, or not bound to this plan */
+    PSA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+    PSA_ERR_TIMEOUT = 5,     /* device: a bounded wait expired; outputs of that block unwritten */
+    PSA_ERR_BOUNDS = 6       /* device: an index outside its table was met and skipped */
+} psa_status_t;
+
+enum { PSA_OUT_BF16 = 0, PSA_OUT_F32 = 1 };
+
+typedef struct {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;   /* 64 or 128 */
+    int32_t page_size;  /* tokens per page of the suffix pool: 16 */
+    float   sm_scale;   /* multiplies q.k before the softmax; > 0 */
+    int32_t out_dtype;  /* PSA_OUT_BF16 or PSA_OUT_F32 */
+    int32_t num_sms;    /* SMs to plan for; 0 = ask the current CUDA device */
+    int32_t reserved;   /* must be 0 */
+} psa_config_t;
+
+/* What the planner decided; for tests, logs and roofline accounting. */
+typedef struct {
+    int32_t num_sms;
+    int32_t num_samples;          /* B */
+    int32_t num_prefix_items;     /* prefix work items (one thread block each) */
+    int32_t num_suffix_items;     /* suffix work items at the planned suffix lengths */
+    int32_t prefix_tile_keys;     /* keys per tensor-core tile (128) */
+    int32_t prefix_tiles_per_item;/* upper bound of key tiles in one prefix item */
+    int32_t suffix_chunk_tokens;  /* tokens per suffix work item */
+    int32_t kernel_launches;      /* device launches one psa_decode enqueues */
+    int64_t num_partial_rows;     /* rows of the partial-result arrays in the workspace */
+} psa_plan_info_t;
+
+/*
+ * Plan stage (part 4 of the design; the paper's "one prompt, many samples" shape is its
+ * only input).  Host only; touches CUDA only when cfg->num_sms == 0.
+ *   prefix_lens [num_prefixes] host: L_p >= 0.
+ *   n_samples_per_prefix [num_prefixes] host: N_p >= 0; B = sum N_p.
+ *   suffix_lens [B] host: upper bounds of S_s used to size the work lists.  psa_decode
+ *     reads the actual lengths from device memory; each must be <= its bound here.
+ * On success *out_plan is a new plan the caller destroys with psa_plan_destroy.
+ */
+psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes,
+                             const int32_t *prefix_lens, const int32_t *n_samples_per_prefix,
+                             const int32_t *suffix_lens, psa_plan_t **out_plan);
+psa_status_t psa_plan_destroy(psa_plan_t *plan);
+psa_status_t psa_plan_get_info(const psa_plan_t *plan, psa_plan_info_t *info);
+
+/* Bytes of device workspace psa_decode needs with this plan (work lists + partial results). */
+size_t psa_plan_workspace_bytes(const psa_plan_t *plan);
+
+/*
+ * Copy the plan's work lists into `workspace` (device, 256-byte aligned, at least
+ * psa_plan_workspace_bytes) and clear its status word.  Enqueued on `cuda_stream`
+ * (a cudaStream_t; NULL = default stream).  Call once per (plan, workspace) pair, before
+ * the first psa_decode that uses them and before any stream capture.
+ */
+psa_status_t psa_plan_bind_workspace(const psa_plan_t *plan, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream);
+
+/*
+ * Host copies of the work lists, for tests.  Each prefix item is 8 int32:
+ *   {first_token (index into the packed prefix), n_keys, kv_head, first_sample,
+ *    n_rows (valid query rows = samples x G), partial_row0, prompt, split}
+ * each suffix item 4 int32: {sample, kv_head, first_token, partial_row0}.
+ * Pass NULL to query the count only.  Returns the number of items.
+ */
+int32_t psa_plan_prefix_items(const psa_plan_t *plan, int32_t *items8);
+int32_t psa_plan_suffix_items(const psa_plan_t *plan, int32_t *items4);
+
+/*
+ * One decode step (prefix, suffix and merge stages).  Only enqueues work on
+ * `cuda_stream`; never synchronises, never allocates device memory.
+ *
+ *   q              [B, Hq, D] bf16 device, contiguous, 16-byte aligned.
+ *   prefix_k/v     bf16 device, 16-byte aligned; element (token t, kv head, d) at
+ *                  t*prefix_strides[0] + head*prefix_strides[1] + d  (elements; D contiguous;
+ *                  strides multiples of 8 elements).  May be NULL when every L_p == 0.
+ *   suffix_k/v_pool bf16 device, 16-byte aligned; element (page, kv head, slot, d) at
+ *                  page*pool_strides[0] + head*pool_strides[1] + slot*pool_strides[2] + d.
+ *   page_indptr    [B+1] int32 device: sample s owns page_indices[page_indptr[s] .. page_indptr[s+1]).
+ *   page_indices   int32 device: physical page ids; token t of sample s is in its page t/16, slot t%16.
+ *   suffix_lens    [B] int32 device: actual S_s, each <= the planned bound (larger is clamped).
+ *   out            [B, Hq, D] device, bf16 or f32 per cfg.out_dtype.
+ *   lse            [B, Hq] f32 device, natural logarithm; -inf for an empty context (out = 0).
+ *   workspace      the buffer bound with psa_plan_bind_workspace.
+ * Concurrent calls must use distinct workspaces.
+ */
+psa_status_t psa_decode(const psa_plan_t *plan, const void *q,
+                        const void *prefix_k, const void *prefix_v, const int64_t prefix_strides[2],
+                        const void *suffix_k_pool, const void *suffix_v_pool, const int64_t pool_strides[3],
+                        const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
+                        void *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The stages one by one, for tests and per-kernel timing.  Same arguments as psa_decode.
+ * prefix and suffix write partial results into the workspace; merge reads them.
+ */
+psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,
+                               const int64_t prefix_strides[2], void *workspace, size_t workspace_bytes,
+                               void *cuda_stream);
+psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void *suffix_k_pool,
+                               const void *suffix_v_pool, const int64_t pool_strides[3],
+                               const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+psa_status_t psa_decode_merge(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The same step with every tensor in HOST memory (pinned memory makes the copies
+ * asynchronous): copies the inputs into `staging` (device, psa_decode_host_staging_bytes),
+ * runs psa_decode, copies out and lse back to the host buffers, all on `cuda_stream`.
+ * num_prefix_tokens / num_pool_pages size the copies; the K/V layouts are the dense
+ * defaults ([tokens, Hkv, D] and [pages, Hkv, 16, D]).  Does not synchronise.
+ */
+size_t psa_decode_host_staging_bytes(const psa_plan_t *plan, int64_t num_prefix_tokens, int64_t num_pool_pages,
+                                     int64_t num_page_indices);
+psa_status_t psa_decode_host(const psa_plan_t *plan, const void *q_host,
+                             const void *prefix_k_host, const void *prefix_v_host, int64_t num_prefix_tokens,
+                             const void *suffix_k_pool_host, const void *suffix_v_pool_host, int64_t num_pool_pages,
+                             const int32_t *page_indptr_host, const int32_t *page_indices_host,
+                             int64_t num_page_indices, const int32_t *suffix_lens_host,
+                             void *out_host, float *lse_host, void *staging, size_t staging_bytes,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Synchronise `cuda_stream` and return the device-side status word of `workspace`
+ * (PSA_OK, PSA_ERR_TIMEOUT or PSA_ERR_BOUNDS), then clear it.
+ */
+psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cuda_stream);
+
+const char *psa_status_string(psa_status_t status);
+const char *psa_last_error_message(void); /* thread-local detail of the last non-OK return */
+int32_t psa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSA_H_ */

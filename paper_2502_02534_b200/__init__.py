@@ -1,0 +1,9 @@
+"""Thin Python binding of the psa C library (``include/psa.h``): argument marshalling only.
+
+Every step of the path runs in the CUDA library.  There is no fallback: if
+``libpsa.so`` has not been built, or no CUDA device is present when a kernel is
+requested, the call raises.
+"""
+from .binding import (  # noqa: F401
+    PsaError, Plan, PlanInfo, decode, decode_host, library, library_path, status_string, EXPORTED_SYMBOLS,
+)

@@ -1,0 +1,250 @@
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
+from dataclasses import dataclass
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_LIB_PATH = _HERE / "libpsa.so"
+_lib = None
+
+PSA_OUT_BF16, PSA_OUT_F32 = 0, 1
+
+# every symbol include/psa.h declares
+EXPORTED_SYMBOLS = [
+    "psa_plan_create", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
+    "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
+    "psa_decode", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status",
+    "psa_status_string", "psa_last_error_message", "psa_version",
+]
+
+
+class PsaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"psa status {status} ({status_string(status)}): {message}")
+        self.status = status
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("num_q_heads", c_int32), ("num_kv_heads", c_int32), ("head_dim", c_int32), ("page_size", c_int32),
+                ("sm_scale", c_float), ("out_dtype", c_int32), ("num_sms", c_int32), ("reserved", c_int32)]
+
+
+class _Info(ctypes.Structure):
+    _fields_ = [("num_sms", c_int32), ("num_samples", c_int32), ("num_prefix_items", c_int32),
+                ("num_suffix_items", c_int32), ("prefix_tile_keys", c_int32), ("prefix_tiles_per_item", c_int32),
+                ("suffix_chunk_tokens", c_int32), ("kernel_launches", c_int32), ("num_partial_rows", c_int64)]
+
+
+@dataclass
+class PlanInfo:
+    num_sms: int
+    num_samples: int
+    num_prefix_items: int
+    num_suffix_items: int
+    prefix_tile_keys: int
+    prefix_tiles_per_item: int
+    suffix_chunk_tokens: int
+    kernel_launches: int
+    num_partial_rows: int
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def library():
+    """Load libpsa.so.  Raises if it has not been built: there is no other implementation."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2502_02534_b200.build`")
+        lib = ctypes.CDLL(str(_LIB_PATH))
+        P = c_void_p
+        lib.psa_plan_create.restype = c_int32
+        lib.psa_plan_create.argtypes = [POINTER(_Config), c_int32, P, P, P, POINTER(c_void_p)]
+        lib.psa_plan_destroy.restype = c_int32
+        lib.psa_plan_destroy.argtypes = [P]
+        lib.psa_plan_get_info.restype = c_int32
+        lib.psa_plan_get_info.argtypes = [P, POINTER(_Info)]
+        lib.psa_plan_workspace_bytes.restype = c_size_t
+        lib.psa_plan_workspace_bytes.argtypes = [P]
+        lib.psa_plan_bind_workspace.restype = c_int32
+        lib.psa_plan_bind_workspace.argtypes = [P, P, c_size_t, P]
+        lib.psa_plan_prefix_items.restype = c_int32
+        lib.psa_plan_prefix_items.argtypes = [P, P]
+        lib.psa_plan_suffix_items.restype = c_int32
+        lib.psa_plan_suffix_items.argtypes = [P, P]
+        lib.psa_decode.restype = c_int32
+        lib.psa_decode.argtypes = [P, P, P, P, POINTER(c_int64), P, P, POINTER(c_int64), P, P, P, P, P, P, c_size_t, P]
+        lib.psa_decode_prefix.restype = c_int32
+        lib.psa_decode_prefix.argtypes = [P, P, P, P, POINTER(c_int64), P, c_size_t, P]
+        lib.psa_decode_suffix.restype = c_int32
+        lib.psa_decode_suffix.argtypes = [P, P, P, P, POINTER(c_int64), P, P, P, P, c_size_t, P]
+        lib.psa_decode_merge.restype = c_int32
+        lib.psa_decode_merge.argtypes = [P, P, P, P, P, c_size_t, P]
+        lib.psa_decode_host_staging_bytes.restype = c_size_t
+        lib.psa_decode_host_staging_bytes.argtypes = [P, c_int64, c_int64, c_int64]
+        lib.psa_decode_host.restype = c_int32
+        lib.psa_decode_host.argtypes = [P, P, P, P, c_int64, P, P, c_int64, P, P, c_int64, P, P, P, P, c_size_t, P, c_size_t, P]
+        lib.psa_check_status.restype = c_int32
+        lib.psa_check_status.argtypes = [P, P, P]
+        lib.psa_status_string.restype = c_char_p
+        lib.psa_status_string.argtypes = [c_int32]
+        lib.psa_last_error_message.restype = c_char_p
+        lib.psa_last_error_message.argtypes = []
+        lib.psa_version.restype = c_int32
+        lib.psa_version.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return library().psa_status_string(int(status)).decode()
+
+
+def _check(status: int):
+    if status != 0:
+        raise PsaError(status, library().psa_last_error_message().decode())
+
+
+def _ptr(t):
+    """Address of a torch tensor / numpy array / None."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+class Plan:
+    """psa_plan_create / psa_plan_destroy, plus the workspace the plan needs (a torch uint8 tensor)."""
+
+    def __init__(self, prefix_lens, n_samples_per_prefix, suffix_lens, *, num_q_heads, num_kv_heads, head_dim,
+                 page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0):
+        lib = library()
+        self.prefix_lens, self.n_samples, self.suffix_len_bounds = _i32(prefix_lens), _i32(n_samples_per_prefix), _i32(suffix_lens)
+        self.num_q_heads, self.num_kv_heads, self.head_dim, self.page_size = num_q_heads, num_kv_heads, head_dim, page_size
+        self.sm_scale = float(sm_scale if sm_scale is not None else head_dim ** -0.5)
+        self.out_dtype = {"bf16": PSA_OUT_BF16, "f32": PSA_OUT_F32}[out_dtype]
+        cfg = _Config(num_q_heads, num_kv_heads, head_dim, page_size, self.sm_scale, self.out_dtype, num_sms, 0)
+        handle = c_void_p()
+        self._h = None
+        _check(lib.psa_plan_create(ctypes.byref(cfg), len(self.prefix_lens), _ptr(self.prefix_lens), _ptr(self.n_samples),
+                                   _ptr(self.suffix_len_bounds), ctypes.byref(handle)))
+        self._h = handle
+        self.workspace = None
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            library().psa_plan_destroy(self._h)
+            self._h = None
+
+    @property
+    def handle(self):
+        return self._h
+
+    @property
+    def info(self) -> PlanInfo:
+        i = _Info()
+        _check(library().psa_plan_get_info(self._h, ctypes.byref(i)))
+        return PlanInfo(*(getattr(i, f[0]) for f in _Info._fields_))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(library().psa_plan_workspace_bytes(self._h))
+
+    def prefix_items(self) -> np.ndarray:
+        n = library().psa_plan_prefix_items(self._h, None)
+        a = np.zeros((n, 8), dtype=np.int32)
+        library().psa_plan_prefix_items(self._h, _ptr(a))
+        return a
+
+    def suffix_items(self) -> np.ndarray:
+        n = library().psa_plan_suffix_items(self._h, None)
+        a = np.zeros((n, 4), dtype=np.int32)
+        library().psa_plan_suffix_items(self._h, _ptr(a))
+        return a
+
+    def bind_workspace(self, workspace=None, stream=None):
+        """Allocate (through torch) or adopt a device workspace and upload the work lists into it."""
+        import torch
+        if workspace is None:
+            workspace = torch.empty(max(256, self.workspace_bytes), dtype=torch.uint8, device="cuda")
+        _check(library().psa_plan_bind_workspace(self._h, _ptr(workspace), workspace.numel(), _stream_ptr(stream)))
+        self.workspace = workspace
+        return workspace
+
+    def check_status(self, stream=None):
+        _check(library().psa_check_status(self._h, _ptr(self.workspace), _stream_ptr(stream)))
+
+
+def _strides(values, n):
+    arr = (c_int64 * n)(*[int(v) for v in values])
+    return arr
+
+
+def default_prefix_strides(plan: Plan):
+    return (plan.num_kv_heads * plan.head_dim, plan.head_dim)
+
+
+def default_pool_strides(plan: Plan):
+    return (plan.num_kv_heads * plan.page_size * plan.head_dim, plan.page_size * plan.head_dim, plan.head_dim)
+
+
+def decode(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,
+           out, lse, *, prefix_strides=None, pool_strides=None, stream=None, stage="all"):
+    """psa_decode (or one of its stages) on torch CUDA tensors.  Only enqueues work."""
+    lib = library()
+    if plan.workspace is None:
+        plan.bind_workspace(stream=stream)
+    ws, wsb, st = _ptr(plan.workspace), plan.workspace.numel(), _stream_ptr(stream)
+    pst = _strides(prefix_strides or default_prefix_strides(plan), 2)
+    qst = _strides(pool_strides or default_pool_strides(plan), 3)
+    if stage == "all":
+        _check(lib.psa_decode(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, _ptr(suffix_k_pool),
+                              _ptr(suffix_v_pool), qst, _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens),
+                              _ptr(out), _ptr(lse), ws, wsb, st))
+    elif stage == "prefix":
+        _check(lib.psa_decode_prefix(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, ws, wsb, st))
+    elif stage == "suffix":
+        _check(lib.psa_decode_suffix(plan.handle, _ptr(q), _ptr(suffix_k_pool), _ptr(suffix_v_pool), qst,
+                                     _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens), ws, wsb, st))
+    elif stage == "merge":
+        _check(lib.psa_decode_merge(plan.handle, _ptr(suffix_lens), _ptr(out), _ptr(lse), ws, wsb, st))
+    else:
+        raise ValueError(stage)
+
+
+def decode_host(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,
+                out, lse, staging, *, stream=None):
+    """psa_decode_host: every tensor is a host buffer (numpy array or pinned torch CPU tensor)."""
+    lib = library()
+    if plan.workspace is None:
+        plan.bind_workspace(stream=stream)
+    n_tok = int(prefix_k.shape[0]) if prefix_k is not None else 0
+    n_pages = int(suffix_k_pool.shape[0]) if suffix_k_pool is not None else 0
+    n_idx = int(page_indices.shape[0]) if page_indices is not None else 0
+    _check(lib.psa_decode_host(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), n_tok, _ptr(suffix_k_pool),
+                               _ptr(suffix_v_pool), n_pages, _ptr(page_indptr), _ptr(page_indices), n_idx,
+                               _ptr(suffix_lens), _ptr(out), _ptr(lse), _ptr(staging), staging.numel(),
+                               _ptr(plan.workspace), plan.workspace.numel(), _stream_ptr(stream)))
+
+
+def host_staging_bytes(plan: Plan, n_prefix_tokens: int, n_pool_pages: int, n_page_indices: int) -> int:
+    return int(library().psa_decode_host_staging_bytes(plan.handle, n_prefix_tokens, n_pool_pages, n_page_indices))

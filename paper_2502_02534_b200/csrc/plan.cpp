@@ -1,0 +1,229 @@
+// Planner: cuts the prefix and suffix stages into work items that fill every SM.
+// Host only, integer arithmetic only.
+//
+// The shape it plans for is the paper's parallel-sampling step (Algorithm 1): a few
+// prompts, each sampled N_p times, so that the N_p * G query rows of a KV head share
+// the prompt's K/V.  Prefix work is counted in (key tile x row group) steps, suffix
+// work in tokens; both cost models charge a fixed start-up per item so that very
+// small pieces are not preferred.
+#include <algorithm>
+#include <cstring>
+#include <limits>
+
+#include "psa_internal.h"
+
+namespace psa {
+namespace {
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Prefix: every (prompt, kv head, row group) streams ceil(L_p / 128) key tiles.  With at
+// most T tiles per item the stage takes ceil(items / SMs) waves of (T + overhead) tile
+// steps; pick the T with the smallest estimate, preferring larger T on ties (fewer
+// partial results to write and merge).
+int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::vector<int64_t> &groups, int num_sms)
+{
+    int64_t max_tiles = 0;
+    for (int64_t t : tiles) max_tiles = std::max(max_tiles, t);
+    if (max_tiles == 0) return 1;
+    const double overhead = 2.0;  // prologue + epilogue of one item, in tile steps
+    double best_cost = std::numeric_limits<double>::infinity();
+    int best_T = 1;
+    for (int64_t T = 1; T <= max_tiles; ++T) {
+        int64_t items = 0, longest = 0;
+        for (size_t p = 0; p < tiles.size(); ++p) {
+            if (tiles[p] == 0) continue;
+            int64_t splits = ceil_div(tiles[p], T);
+            items += groups[p] * splits;
+            longest = std::max(longest, ceil_div(tiles[p], splits));
+        }
+        int64_t waves = ceil_div(items, num_sms);
+        double cost = double(waves) * (double(longest) + overhead);
+        if (cost <= best_cost) { best_cost = cost; best_T = int(T); }
+    }
+    return best_T;
+}
+
+// Suffix: items are dispatched greedily to 2 resident blocks per SM.  Estimate =
+// (sum of item costs) / slots + cost of one full item (the tail); cost = tokens + 64.
+int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sms)
+{
+    const double overhead = 64.0;
+    const double slots = 2.0 * num_sms;
+    double best_cost = std::numeric_limits<double>::infinity();
+    int best = 64;
+    for (int C = 64; C <= 8192; C *= 2) {
+        double sum = 0.0;
+        int64_t longest = 0;
+        for (int s = 0; s < n; ++s) {
+            int64_t S = lens[s];
+            if (S <= 0) continue;
+            int64_t chunks = ceil_div(S, C);
+            sum += double(num_kv_heads) * (double(S) + overhead * double(chunks));
+            longest = std::max<int64_t>(longest, std::min<int64_t>(S, C));
+        }
+        double cost = sum / slots + double(longest) + overhead;
+        if (cost < best_cost) { best_cost = cost; best = C; }
+    }
+    return best;
+}
+
+}  // namespace
+
+psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefix_lens, const int32_t *n_samples,
+                        const int32_t *suffix_lens, psa_plan *plan, std::string *err)
+{
+    auto fail = [&](psa_status_t st, const char *msg) { if (err) *err = msg; return st; };
+    if (cfg.num_q_heads <= 0 || cfg.num_kv_heads <= 0 || cfg.num_q_heads % cfg.num_kv_heads != 0)
+        return fail(PSA_ERR_INVALID_ARG, "num_q_heads must be a positive multiple of num_kv_heads");
+    const int G = cfg.num_q_heads / cfg.num_kv_heads;
+    if (cfg.head_dim != 64 && cfg.head_dim != 128) return fail(PSA_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    if (G != 1 && G != 2 && G != 4 && G != 8) return fail(PSA_ERR_UNSUPPORTED, "group size must be 1, 2, 4 or 8");
+    if (cfg.page_size != kPageSize) return fail(PSA_ERR_UNSUPPORTED, "page_size must be 16");
+    if (!(cfg.sm_scale > 0.0f) || !(cfg.sm_scale < std::numeric_limits<float>::infinity()))
+        return fail(PSA_ERR_INVALID_ARG, "sm_scale must be positive and finite");
+    if (cfg.out_dtype != PSA_OUT_BF16 && cfg.out_dtype != PSA_OUT_F32)
+        return fail(PSA_ERR_UNSUPPORTED, "out_dtype must be PSA_OUT_BF16 or PSA_OUT_F32");
+    if (cfg.reserved != 0) return fail(PSA_ERR_INVALID_ARG, "reserved must be 0");
+    if (cfg.num_sms <= 0) return fail(PSA_ERR_INVALID_ARG, "num_sms must be positive here");
+    if (P < 0 || (P > 0 && (!prefix_lens || !n_samples))) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
+
+    plan->cfg = cfg;
+    plan->group = G;
+    plan->num_prefixes = P;
+    plan->prefix_lens.assign(prefix_lens, prefix_lens + P);
+    plan->n_samples.assign(n_samples, n_samples + P);
+    int64_t B = 0, total_tokens = 0;
+    for (int p = 0; p < P; ++p) {
+        if (prefix_lens[p] < 0 || n_samples[p] < 0) return fail(PSA_ERR_INVALID_ARG, "negative length or sample count");
+        B += n_samples[p];
+        total_tokens += prefix_lens[p];
+    }
+    if (B > (1 << 24) || total_tokens > (int64_t(1) << 30)) return fail(PSA_ERR_UNSUPPORTED, "problem too large");
+    if (B > 0 && !suffix_lens) return fail(PSA_ERR_INVALID_ARG, "null suffix_lens");
+    for (int64_t s = 0; s < B; ++s)
+        if (suffix_lens[s] < 0 || suffix_lens[s] > (1 << 24)) return fail(PSA_ERR_INVALID_ARG, "suffix length out of range");
+    plan->num_samples = int32_t(B);
+    plan->total_prefix_tokens = total_tokens;
+    plan->suffix_len_bounds.assign(suffix_lens, suffix_lens + B);
+
+    // ---- prefix items
+    const int samples_per_group = kPrefixRowsPerItem / G;  // samples in one 256-row group
+    std::vector<int64_t> tiles(P), groups(P);
+    for (int p = 0; p < P; ++p) {
+        tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;
+        groups[p] = int64_t(cfg.num_kv_heads) * ceil_div(n_samples[p], samples_per_group);
+    }
+    const int T = choose_prefix_tiles_per_item(tiles, groups, cfg.num_sms);
+    plan->prefix_tiles_per_item = T;
+
+    plan->sample_info.assign(size_t(B), SampleInfo{});
+    plan->prefix_items.clear();
+    int64_t next_row = 0;  // partial rows are handed out prefix first, then suffix
+    int64_t tok_off = 0, samp_off = 0;
+    int longest_item_tiles = 0;
+    for (int p = 0; p < P; ++p) {
+        const int64_t N = n_samples[p], L = prefix_lens[p], R = N * G;
+        const int64_t splits = tiles[p] > 0 ? ceil_div(tiles[p], T) : 0;
+        const int64_t base = next_row;
+        for (int64_t i = 0; i < N; ++i) {
+            SampleInfo &si = plan->sample_info[size_t(samp_off + i)];
+            si.pre_row0 = int32_t(base + i * G);
+            si.pre_split_stride = int32_t(R);
+            si.pre_splits = int32_t(splits);
+            si.pre_head_stride = int32_t(R * splits);
+            si.prompt = p;
+        }
+        if (splits > 0) {
+            // key tiles are dealt out as evenly as possible: the first `extra` splits get one more
+            const int64_t per = tiles[p] / splits, extra = tiles[p] % splits;
+            for (int kv = 0; kv < cfg.num_kv_heads; ++kv) {
+                int64_t tile0 = 0;
+                for (int64_t j = 0; j < splits; ++j) {
+                    const int64_t nt = per + (j < extra ? 1 : 0);
+                    const int64_t key0 = tile0 * kPrefixTileKeys;
+                    const int64_t key1 = std::min<int64_t>(L, (tile0 + nt) * kPrefixTileKeys);
+                    longest_item_tiles = std::max<int>(longest_item_tiles, int(nt));
+                    for (int64_t s0 = 0; s0 < N; s0 += samples_per_group) {
+                        PrefixItem it;
+                        it.first_token = int32_t(tok_off + key0);
+                        it.n_keys = int32_t(key1 - key0);
+                        it.kv_head = kv;
+                        it.first_sample = int32_t(samp_off + s0);
+                        it.n_rows = int32_t(std::min<int64_t>(samples_per_group, N - s0) * G);
+                        it.partial_row0 = int32_t(base + (int64_t(kv) * splits + j) * R + s0 * G);
+                        it.prompt = p;
+                        it.split = int32_t(j);
+                        plan->prefix_items.push_back(it);
+                    }
+                    tile0 += nt;
+                }
+            }
+            next_row += int64_t(cfg.num_kv_heads) * splits * R;
+        }
+        tok_off += L;
+        samp_off += N;
+    }
+    plan->prefix_tiles_per_item = std::max(1, longest_item_tiles);
+    // longest items first: the hardware scheduler then fills the tail with short ones
+    std::stable_sort(plan->prefix_items.begin(), plan->prefix_items.end(), [](const PrefixItem &a, const PrefixItem &b) {
+        const int64_t ca = int64_t(ceil_div(a.n_keys, kPrefixTileKeys)) * (a.n_rows > kPrefixTileRows ? 2 : 1);
+        const int64_t cb = int64_t(ceil_div(b.n_keys, kPrefixTileKeys)) * (b.n_rows > kPrefixTileRows ? 2 : 1);
+        return ca > cb;
+    });
+
+    // ---- suffix items
+    const int C = choose_suffix_chunk(suffix_lens, int(B), cfg.num_kv_heads, cfg.num_sms);
+    plan->suffix_chunk_tokens = C;
+    plan->suffix_items.clear();
+    for (int64_t s = 0; s < B; ++s) {
+        SampleInfo &si = plan->sample_info[size_t(s)];
+        const int64_t S = suffix_lens[s];
+        const int64_t chunks = ceil_div(S, C);
+        si.suf_row0 = int32_t(next_row);
+        si.suf_chunks = int32_t(chunks);
+        si.suf_len_bound = int32_t(S);
+        for (int kv = 0; kv < cfg.num_kv_heads; ++kv)
+            for (int64_t c = 0; c < chunks; ++c) {
+                SuffixItem it;
+                it.sample = int32_t(s);
+                it.kv_head = kv;
+                it.first_token = int32_t(c * C);
+                it.partial_row0 = int32_t(next_row + (int64_t(kv) * chunks + c) * G);
+                plan->suffix_items.push_back(it);
+            }
+        next_row += int64_t(cfg.num_kv_heads) * chunks * G;
+    }
+    // full chunks first, ragged last chunks after them (longest first)
+    std::stable_sort(plan->suffix_items.begin(), plan->suffix_items.end(), [&](const SuffixItem &a, const SuffixItem &b) {
+        const int la = std::min<int>(C, suffix_lens[a.sample] - a.first_token);
+        const int lb = std::min<int>(C, suffix_lens[b.sample] - b.first_token);
+        return la > lb;
+    });
+    if (next_row >= (int64_t(1) << 31)) return fail(PSA_ERR_UNSUPPORTED, "too many partial rows");
+    plan->num_partial_rows = next_row;
+
+    // ---- workspace layout and the host image of the lists
+    WorkspaceLayout &ws = plan->ws;
+    size_t off = 0;
+    ws.status_off = off;          off = align_up(off + sizeof(int32_t) * kStatusWords, 256);
+    ws.prefix_items_off = off;    off = align_up(off + sizeof(PrefixItem) * plan->prefix_items.size(), 256);
+    ws.suffix_items_off = off;    off = align_up(off + sizeof(SuffixItem) * plan->suffix_items.size(), 256);
+    ws.sample_info_off = off;     off = align_up(off + sizeof(SampleInfo) * plan->sample_info.size(), 256);
+    ws.lists_end = off;
+    ws.partial_lse_off = off;     off = align_up(off + sizeof(float) * size_t(next_row), 256);
+    ws.partial_o_off = off;       off = align_up(off + sizeof(float) * size_t(next_row) * size_t(cfg.head_dim), 256);
+    ws.total = off;
+
+    plan->upload.assign(ws.lists_end, 0);
+    if (!plan->prefix_items.empty())
+        std::memcpy(plan->upload.data() + ws.prefix_items_off, plan->prefix_items.data(), sizeof(PrefixItem) * plan->prefix_items.size());
+    if (!plan->suffix_items.empty())
+        std::memcpy(plan->upload.data() + ws.suffix_items_off, plan->suffix_items.data(), sizeof(SuffixItem) * plan->suffix_items.size());
+    if (!plan->sample_info.empty())
+        std::memcpy(plan->upload.data() + ws.sample_info_off, plan->sample_info.data(), sizeof(SampleInfo) * plan->sample_info.size());
+    return PSA_OK;
+}
+
+}  // namespace psa

@@ -1,0 +1,516 @@
+// Prefix stage: every sample's query rows of one KV head, batched against the shared
+// prompt K/V, on the 5th-generation tensor cores (tcgen05) with accumulators in tensor
+// memory (TMEM) and operands brought in by TMA.
+//
+// Arithmetic: the paper's attn Task 2 recurrence (deferred division).  For one key tile
+// with raw scores s = q.k and c = sm_scale * log2(e):
+//     m' = max(m, max_j c*s_j),  p_j = 2^(c*s_j - m'),  l' = l * 2^(m - m') + sum_j p_j,
+//     O' = O * 2^(m - m') + P V,      and at the end  out = O / l,  lse = (m + log2 l) ln 2.
+// The reference maximum is only moved when a tile's maximum exceeds it by more than 2^8
+// (the result is unchanged: the factor cancels between O and l), so the accumulator in
+// TMEM is almost never rescaled.
+//
+// One thread block = one work item = (kv head, up to 256 query rows, a range of keys):
+//   warps 0-3   softmax warpgroup of row tile 0 (rows 0..127; thread = TMEM lane = row)
+//   warps 4-7   softmax warpgroup of row tile 1 (rows 128..255; idle when the item has <= 128 rows)
+//   warp  8     TMA producer: Q once, then K and V tiles of 128 keys through a ring of buffers
+//   warp  9     MMA issuer (one elected lane) and owner of the TMEM allocation
+// Per key tile and row tile:  S = Q K^T (SS MMA, K-major operands, 128-byte swizzle)
+// -> softmax warpgroup reads S from TMEM, writes P (bf16) over it -> O += P V (TS MMA,
+// P from TMEM, V as MN-major B operand).  The two row tiles alternate on the tensor pipe,
+// so one tile's softmax overlaps the other's MMAs; K/V are read from HBM/L2 once per item.
+//
+// Every wait on an mbarrier is bounded: when the limit passes, the block raises
+// PSA_ERR_TIMEOUT in the status word, stops storing results, and drains to a normal exit
+// (TMEM freed) instead of spinning.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "psa_internal.h"
+
+namespace psa {
+namespace {
+
+constexpr int kSoftmaxWarps = 8;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kThreads = 10 * 32;
+constexpr int kRing = 5;                 // K/V tile buffers in flight
+constexpr float kRescaleThreshold = 8.f; // log2 units
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit passed or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread = lane (row), register i = column i
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// ---------------------------------------------------------------- descriptors
+// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte
+// offsets (all in 16-byte units), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= uint64_t((addr >> 4) & 0x3FFFu);
+    d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= uint64_t(1) << 46;   // version
+    d |= uint64_t(2) << 61;   // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor for kind::f16: bf16 x bf16 -> f32, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
+{
+    return (1u << 4) /* D = f32 */ | (1u << 7) /* A = bf16 */ | (1u << 10) /* B = bf16 */ |
+           (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+}
+
+template <int D>
+struct PrefixSmem {
+    static constexpr int kHalfBytes = kPrefixTileKeys * 128;          // one TMA box: 128 rows x 64 bf16
+    static constexpr int kHalves = D / 64;
+    static constexpr int kTileBytes = kHalves * kHalfBytes;           // a Q, K or V tile
+    static constexpr int kQOff = 0;                                   // 2 Q tiles
+    static constexpr int kRingOff = 2 * kTileBytes;
+    static constexpr int kBarOff = kRingOff + kRing * kTileBytes;
+    static constexpr int kNumBars = 1 + 2 * kRing + 6;               // q, full[], empty[], s_full[2], p_full[2], o_done[2]
+    static constexpr int kTmemPtrOff = kBarOff + 8 * kNumBars;
+    static constexpr int kAbortOff = kTmemPtrOff + 4;
+    static constexpr int kTotal = kAbortOff + 4 + 1024;               // + slack to align the base to 1024
+    static constexpr int kTmemCols = 512;                             // S0 S1 (128 each) at 0, O0 O1 (D each) at 256
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+              const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
+              float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+{
+    using L = PrefixSmem<D>;
+    constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
+    constexpr int kPSteps = kPrefixTileKeys / 16;   // MMA k-steps of PV
+    constexpr uint32_t kIdescQK = make_idesc(kPrefixTileKeys, false);
+    constexpr uint32_t kIdescPV = make_idesc(D, true);
+    constexpr uint32_t kColS = 0, kColO = 2 * kPrefixTileKeys;   // S_t at t*128, O_t at 256 + t*D
+
+    extern __shared__ unsigned char smem_unaligned[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_unaligned) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::kBarOff;
+    auto bar_q = [&]() { return bar0; };
+    auto bar_full = [&](int i) { return bar0 + 8 * (1 + i); };
+    auto bar_empty = [&](int i) { return bar0 + 8 * (1 + kRing + i); };
+    auto bar_s = [&](int t) { return bar0 + 8 * (1 + 2 * kRing + t); };
+    auto bar_p = [&](int t) { return bar0 + 8 * (3 + 2 * kRing + t); };
+    auto bar_o = [&](int t) { return bar0 + 8 * (5 + 2 * kRing + t); };
+    volatile uint32_t *tmem_ptr = reinterpret_cast<volatile uint32_t *>(smem + L::kTmemPtrOff);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kAbortOff);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int4 it0 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));
+    const int4 it1 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x) + 1);
+    const int first_token = it0.x, n_keys = it0.y, kv = it0.z, first_sample = it0.w;
+    const int n_rows = it1.x, prow0 = it1.y;
+    const int n_tiles = (n_keys + kPrefixTileKeys - 1) / kPrefixTileKeys;
+    const int n_slots = n_rows > kPrefixTileRows ? 2 : 1;
+    const int samples_per_tile = kPrefixTileRows / group;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        mbar_init(bar_q(), 1);
+        for (int i = 0; i < kRing; ++i) { mbar_init(bar_full(i), 1); mbar_init(bar_empty(i), 1); }
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128); mbar_init(bar_o(t), 1); }
+        fence_barrier_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_ptr)), L::kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && lane == 0) { prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr;
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(bar_q(), n_slots * L::kTileBytes);
+            for (int t = 0; t < n_slots; ++t)
+                for (int h = 0; h < L::kHalves; ++h)
+                    tma_load_4d(sbase + L::kQOff + t * L::kTileBytes + h * L::kHalfBytes, &map_q, bar_q(), h * 64, 0, kv,
+                                first_sample + t * samples_per_tile);
+            // ring order: K0 V0 K1 V1 ...
+            for (int i = 0; i < 2 * n_tiles; ++i) {
+                const int slot = i % kRing, use = i / kRing;
+                if (use > 0 && !mbar_wait(bar_empty(slot), (use - 1) & 1, abort_flag)) break;
+                const int tok = first_token + (i >> 1) * kPrefixTileKeys;
+                const CUtensorMap *map = (i & 1) ? &map_v : &map_k;
+                mbar_expect_tx(bar_full(slot), L::kTileBytes);
+                for (int h = 0; h < L::kHalves; ++h)
+                    tma_load_3d(sbase + L::kRingOff + slot * L::kTileBytes + h * L::kHalfBytes, map, bar_full(slot), h * 64, kv, tok);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = mbar_wait(bar_q(), 0, abort_flag);
+            auto issue_qk = [&](int t, int j) {   // S_t = Q_t K_j^T ; K_j is ring entry 2j
+                const int slot = (2 * j) % kRing;
+                const uint32_t qa = sbase + L::kQOff + t * L::kTileBytes;
+                const uint32_t kb = sbase + L::kRingOff + slot * L::kTileBytes;
+#pragma unroll
+                for (int k = 0; k < kKSteps; ++k) {
+                    const uint32_t off = (k / 4) * L::kHalfBytes + (k % 4) * 32;
+                    mma_ss(tmem_base + kColS + t * kPrefixTileKeys, make_smem_desc(qa + off, 16, 1024),
+                           make_smem_desc(kb + off, 16, 1024), kIdescQK, k > 0);
+                }
+            };
+            auto issue_pv = [&](int t, int j) {   // O_t += P_t V_j ; V_j is ring entry 2j+1
+                const int slot = (2 * j + 1) % kRing;
+                const uint32_t vb = sbase + L::kRingOff + slot * L::kTileBytes;
+#pragma unroll
+                for (int k = 0; k < kPSteps; ++k)
+                    mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kPrefixTileKeys + k * 8,
+                           make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV, (j > 0 || k > 0));
+            };
+            if (ok) ok = mbar_wait(bar_full(0), 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                for (int t = 0; t < n_slots; ++t) { issue_qk(t, 0); tc_commit(bar_s(t)); }
+            }
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                const int vslot = (2 * j + 1) % kRing, kslot = (2 * j) % kRing;
+                if (!(ok = mbar_wait(bar_full(vslot), ((2 * j + 1) / kRing) & 1, abort_flag))) break;
+                if (j + 1 < n_tiles) {
+                    const int nslot = (2 * j + 2) % kRing;
+                    if (!(ok = mbar_wait(bar_full(nslot), ((2 * j + 2) / kRing) & 1, abort_flag))) break;
+                }
+                for (int t = 0; t < n_slots; ++t) {
+                    if (!(ok = mbar_wait(bar_p(t), j & 1, abort_flag))) break;
+                    tc_fence_after();
+                    issue_pv(t, j);
+                    if (t == n_slots - 1) { tc_commit(bar_empty(kslot)); tc_commit(bar_empty(vslot)); }
+                    if (j + 1 < n_tiles) { issue_qk(t, j + 1); tc_commit(bar_s(t)); }
+                    else tc_commit(bar_o(t));
+                }
+            }
+        }
+    } else if (warp < 4 * n_slots) {
+        // ------------------------------------------------------------ softmax + epilogue
+        const int t = warp >> 2;                       // row tile
+        const int row = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t s_addr = tmem_base + lane_addr + kColS + t * kPrefixTileKeys;
+        const uint32_t o_addr = tmem_base + lane_addr + kColO + t * D;
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        uint32_t sreg[4][32];
+        for (int j = 0; j < n_tiles; ++j) {
+            if (!(ok = mbar_wait(bar_s(t), j & 1, abort_flag))) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
+            tmem_wait_ld();
+            const int valid = n_keys - j * kPrefixTileKeys;   // >= 1; < 128 only on the last tile
+            float tmax = -INFINITY;
+            if (valid >= kPrefixTileKeys) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sreg[c][i]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;   // -inf: masked key
+                        tmax = fmaxf(tmax, __uint_as_float(sreg[c][i]));
+                    }
+            }
+            tmax *= scale_log2;
+            // Move the reference maximum only when needed; the whole warp takes the slow path together
+            // because TMEM loads and stores are warp-collective.
+            const bool need = tmax > m_ref + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+                const float m_new = need ? tmax : m_ref;
+                const float alpha = need ? fast_exp2(m_ref - m_new) : 1.f;   // 0 on the first tile
+                if (j > 0) {
+                    // s_full of tile j was committed after PV of tile j-1: O is quiescent until P of tile j is handed over
+                    uint32_t oreg[32];
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(o_addr + c * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
+                        tmem_st32(o_addr + c * 32, oreg);
+                    }
+                    tmem_wait_st();
+                }
+                l_sum *= alpha;
+                m_ref = m_new;
+            }
+            // p = 2^(c*s - m_ref); row sum from the fp32 values; P packed to bf16 over the first 64 columns of S
+            float psum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_ref));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_ref));
+                    psum += p0 + p1;
+                    sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                }
+            }
+            l_sum += psum;
+            tmem_st32(s_addr, sreg[0]);
+            tmem_st32(s_addr + 32, sreg[1]);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p(t));
+        }
+        // ---- epilogue: out = O / l, lse = (m + log2 l) ln 2
+        if (ok) ok = mbar_wait(bar_o(t), 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            const int r = t * kPrefixTileRows + row;
+            const float inv = 1.f / l_sum;
+            float *dst = partial_o + size_t(prow0 + r) * D;
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t oreg[32];
+                tmem_ld32(o_addr + c * 32, oreg);
+                tmem_wait_ld();
+                if (r < n_rows) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4 *>(dst + c * 32 + i) =
+                            make_float4(__uint_as_float(oreg[i]) * inv, __uint_as_float(oreg[i + 1]) * inv,
+                                        __uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
+                }
+            }
+            if (r < n_rows) partial_lse[prow0 + r] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, int(PSA_ERR_TIMEOUT));
+        // let copies that were already issued land before the block's shared memory is released
+        if (warp == kProducerWarp && lane == 0) {
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 2000000ull) { }
+        }
+        __syncthreads();
+    }
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------- host side
+using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                              const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode_fn(std::string *err)
+{
+    static EncodeFn fn = nullptr;
+    static std::once_flag once;
+    static cudaError_t rc = cudaSuccess;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        rc = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (rc == cudaSuccess && q == cudaDriverEntryPointSuccess) fn = reinterpret_cast<EncodeFn>(p);
+    });
+    if (!fn && err) *err = "cuTensorMapEncodeTiled is not available from the driver";
+    return fn;
+}
+
+bool encode(EncodeFn fn, CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes,
+            const cuuint32_t *box, std::string *err)
+{
+    cuuint32_t elem[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, cuuint32_t(rank), const_cast<void *>(base), dims, strides_bytes, box,
+                    elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        if (err) *err = "cuTensorMapEncodeTiled failed with code " + std::to_string(int(r));
+        return false;
+    }
+    return true;
+}
+
+template <int D>
+int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
+{
+    using L = PrefixSmem<D>;
+    auto kern = prefix_kernel<D>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return int(e);
+        configured = true;
+    }
+    const float scale_log2 = a.sm_scale * 1.4426950408889634f;
+    kern<<<a.num_items, kThreads, L::kTotal, st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, scale_log2,
+                                                   a.partial_o, a.partial_lse, a.status);
+    return int(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
+{
+    if (a.num_items == 0) return 0;
+    EncodeFn fn = get_encode_fn(err);
+    if (!fn) return int(cudaErrorNotSupported);
+    const int G = a.num_q_heads / a.num_kv_heads;
+    const int D = a.head_dim;
+    CUtensorMap mq, mk, mv;
+    {   // Q as (d, g, kv head, sample): a box of (64, G, 1, 128/G) lands as 128 rows ordered sample-major, g fastest
+        const cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(G), cuuint64_t(a.num_kv_heads), cuuint64_t(a.num_samples)};
+        const cuuint64_t strides[3] = {cuuint64_t(D) * 2, cuuint64_t(G) * D * 2, cuuint64_t(a.num_q_heads) * D * 2};
+        const cuuint32_t box[4] = {64, cuuint32_t(G), 1, cuuint32_t(kPrefixTileRows / G)};
+        if (!encode(fn, &mq, a.q, 4, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+    }
+    {   // K and V as (d, kv head, token): a box of (64, 1, 128) is one half of a 128-key tile
+        const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(a.num_kv_heads), cuuint64_t(a.total_tokens)};
+        const cuuint64_t strides[2] = {cuuint64_t(a.stride_head) * 2, cuuint64_t(a.stride_tok) * 2};
+        const cuuint32_t box[3] = {64, 1, cuuint32_t(kPrefixTileKeys)};
+        if (!encode(fn, &mk, a.k, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+        if (!encode(fn, &mv, a.v, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int rc = D == 128 ? launch_one<128>(a, mq, mk, mv, st) : launch_one<64>(a, mq, mk, mv, st);
+    if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));
+    return rc;
+}
+
+}  // namespace psa

@@ -1,0 +1,131 @@
+// Internal declarations shared by the planner, the launchers and the C ABI.
+// Nothing here is part of the public interface (include/psa.h).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "psa.h"
+
+namespace psa {
+
+constexpr int kPageSize = 16;          // tokens per suffix page
+constexpr int kPrefixTileKeys = 128;   // keys per tensor-core tile (N of QK^T, K of PV)
+constexpr int kPrefixTileRows = 128;   // query rows per softmax warpgroup (M of one MMA)
+constexpr int kPrefixRowsPerItem = 256;// two row tiles share the K/V stream of one thread block
+constexpr int kStatusWords = 64;       // int32 words reserved at the start of the workspace
+
+// One thread block of the prefix stage: a (prompt, kv head, row group, key range).
+struct PrefixItem {
+    int32_t first_token;   // index into the packed prefix arrays
+    int32_t n_keys;        // > 0
+    int32_t kv_head;
+    int32_t first_sample;  // sample index of row 0
+    int32_t n_rows;        // valid rows, 1..256 (row = local_sample * G + g)
+    int32_t partial_row0;  // row of the partial arrays that receives row 0
+    int32_t prompt;
+    int32_t split;
+};
+static_assert(sizeof(PrefixItem) == 32, "PrefixItem is read as two int4");
+
+// One thread block of the suffix stage: a (sample, kv head, token chunk).
+struct SuffixItem {
+    int32_t sample;
+    int32_t kv_head;
+    int32_t first_token;   // multiple of the chunk size
+    int32_t partial_row0;  // row of the partial arrays that receives query head g = 0
+};
+static_assert(sizeof(SuffixItem) == 16, "SuffixItem is read as one int4");
+
+// Where the merge stage finds the partial results of one sample.
+// prefix row of (kv head, split j, g): pre_row0 + kv*pre_head_stride + j*pre_split_stride + g
+// suffix row of (kv head, chunk c, g): suf_row0 + (kv*suf_chunks + c)*G + g
+struct SampleInfo {
+    int32_t pre_row0;
+    int32_t pre_split_stride;
+    int32_t pre_splits;
+    int32_t pre_head_stride;
+    int32_t suf_row0;
+    int32_t suf_chunks;     // chunks at the planned suffix length
+    int32_t suf_len_bound;  // planned suffix length
+    int32_t prompt;
+};
+static_assert(sizeof(SampleInfo) == 32, "SampleInfo is read as two int4");
+
+struct WorkspaceLayout {
+    size_t status_off = 0;       // kStatusWords int32
+    size_t prefix_items_off = 0;
+    size_t suffix_items_off = 0;
+    size_t sample_info_off = 0;
+    size_t lists_end = 0;        // bytes copied by bind_workspace
+    size_t partial_lse_off = 0;  // float [num_partial_rows]
+    size_t partial_o_off = 0;    // float [num_partial_rows, D]
+    size_t total = 0;
+};
+
+}  // namespace psa
+
+struct psa_plan {
+    psa_config_t cfg{};
+    int32_t num_prefixes = 0;
+    int32_t num_samples = 0;
+    int32_t group = 1;  // G
+    int64_t total_prefix_tokens = 0;
+    std::vector<int32_t> prefix_lens, n_samples, suffix_len_bounds;
+    std::vector<psa::PrefixItem> prefix_items;
+    std::vector<psa::SuffixItem> suffix_items;
+    std::vector<psa::SampleInfo> sample_info;
+    int32_t prefix_tiles_per_item = 0;
+    int32_t suffix_chunk_tokens = 0;
+    int64_t num_partial_rows = 0;
+    psa::WorkspaceLayout ws;
+    std::vector<unsigned char> upload;  // host image of [0, ws.lists_end)
+};
+
+namespace psa {
+
+// plan.cpp
+psa_status_t build_plan(const psa_config_t &cfg, int32_t num_prefixes, const int32_t *prefix_lens,
+                        const int32_t *n_samples, const int32_t *suffix_lens, psa_plan *plan, std::string *err);
+
+// Launchers (one per .cu file). All enqueue on `stream` and return a CUDA error code (0 = ok).
+struct PrefixArgs {
+    const void *q, *k, *v;
+    int64_t stride_tok, stride_head;  // elements
+    int64_t total_tokens;
+    int32_t num_samples, num_q_heads, num_kv_heads, head_dim;
+    float sm_scale;
+    const PrefixItem *items;  // device
+    int32_t num_items;
+    float *partial_o, *partial_lse;  // device
+    int32_t *status;                 // device
+};
+int launch_prefix(const PrefixArgs &a, void *stream, std::string *err);
+
+struct SuffixArgs {
+    const void *q, *pool_k, *pool_v;
+    int64_t stride_page, stride_head, stride_tok;  // elements
+    const int32_t *page_indptr, *page_indices, *suffix_lens;  // device
+    int32_t num_q_heads, num_kv_heads, head_dim;
+    float sm_scale;
+    const SuffixItem *items;      // device
+    const SampleInfo *sample_info;// device
+    int32_t num_items, chunk_tokens;
+    float *partial_o, *partial_lse;
+    int32_t *status;
+};
+int launch_suffix(const SuffixArgs &a, void *stream, std::string *err);
+
+struct MergeArgs {
+    const SampleInfo *sample_info;  // device
+    const int32_t *suffix_lens;     // device
+    const float *partial_o, *partial_lse;
+    int32_t num_samples, num_q_heads, num_kv_heads, head_dim, chunk_tokens, out_dtype;
+    void *out;
+    float *lse;
+};
+int launch_merge(const MergeArgs &a, void *stream, std::string *err);
+
+}  // namespace psa

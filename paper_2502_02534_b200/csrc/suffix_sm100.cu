@@ -1,0 +1,296 @@
+// Suffix stage: each sample's G query rows (one KV head) against its own generated
+// tokens, stored in 16-token pages scattered through a pool.
+//
+// Arithmetic is the deferred-division online softmax (the paper's attn Task 2
+// recurrence: running maximum m, running sum l, un-normalised accumulator O), applied
+// page by page; the division happens once, when the block writes its partial result.
+//
+// The stage is bound by HBM: every K and V byte is read exactly once and there are only
+// G (<= 8) flops per byte.  Design for that bound:
+//   * one thread block per (sample, kv head, token chunk); its 4 warps take pages
+//     round-robin, each with a private ring of kStages (K page + V page) buffers that
+//     it fills with 16-byte cp.async copies -- a page of one head is 16 x D bf16 =
+//     4 KB contiguous (D = 128), so every copy instruction of a warp reads 512
+//     consecutive bytes.  No block-wide barrier in the main loop.
+//   * the dot products run on warp-level tensor-core MMAs (m16n8k16, bf16 in, fp32
+//     accumulate) with the G query rows padded to 16: plain FMAs could not keep up
+//     with HBM at G = 8.  K fragments come from ldmatrix, V fragments from
+//     ldmatrix.trans, both conflict-free through a 16-byte XOR swizzle of the rows.
+//   * row maxima are refreshed lazily: the quad shuffle + rescale only runs when some
+//     logit exceeds the reference maximum by more than 2^8.
+//   * slots of the last page beyond the sample's length are zero-filled by the copy
+//     (source size 0), never read from memory, and masked to -inf before the softmax.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "psa_internal.h"
+
+namespace psa {
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kStages = 3;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <int D>
+struct SuffixSmem {
+    static constexpr int kRowBytes = D * 2;            // one token of one head
+    static constexpr int kPageBytes = kPageSize * kRowBytes;
+    static constexpr int kStageBytes = 2 * kPageBytes; // K page + V page
+    static constexpr int kWarpBytes = kStages * kStageBytes;
+    static constexpr int kTotal = kWarps * kWarpBytes;
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kWarps * 32, 2)
+suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ pool_k,
+              const __nv_bfloat16 *__restrict__ pool_v, int64_t stride_page, int64_t stride_head, int64_t stride_tok,
+              const int32_t *__restrict__ page_indptr, const int32_t *__restrict__ page_indices,
+              const int32_t *__restrict__ suffix_lens, const SuffixItem *__restrict__ items,
+              const SampleInfo *__restrict__ sample_info, int num_q_heads, int chunk_tokens, float scale_log2,
+              float *__restrict__ partial_o, float *__restrict__ partial_lse)
+{
+    using L = SuffixSmem<D>;
+    constexpr int KK = D / 16;           // k-steps of QK^T
+    constexpr int DN = D / 8;            // n-tiles of PV
+    constexpr int CPR = L::kRowBytes / 16;  // 16-byte chunks per token row
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int4 item = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));
+    const int s = item.x, kv = item.y, tok0 = item.z, prow0 = item.w;
+    int S = __ldg(suffix_lens + s);
+    S = min(S, __ldg(&sample_info[s].suf_len_bound));
+    const int n_tok = min(S - tok0, chunk_tokens);
+    if (n_tok <= 0) return;  // the merge stage derives the chunk count from the same length
+    const int n_pages = (n_tok + kPageSize - 1) / kPageSize;
+    const int my_pages = (n_pages - warp + kWarps - 1) / kWarps;  // pages warp, warp+4, ...
+    const int32_t *my_page_ids = page_indices + __ldg(page_indptr + s) + tok0 / kPageSize;
+
+    // ---- query fragments: rows g < G of a 16-row tile; rows >= G stay zero
+    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
+    uint32_t qa0[KK], qa2[KK];
+    {
+        const __nv_bfloat16 *qp = q + (size_t(s) * num_q_heads + size_t(kv) * G + qrow) * D + qcol;
+#pragma unroll
+        for (int kk = 0; kk < KK; ++kk) {
+            qa0[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16)) : 0u;
+            qa2[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16 + 8)) : 0u;
+        }
+    }
+
+    const uint32_t warp_smem = smem_u32(smem_raw) + warp * L::kWarpBytes;
+    const __nv_bfloat16 *head_k = pool_k + int64_t(kv) * stride_head;
+    const __nv_bfloat16 *head_v = pool_v + int64_t(kv) * stride_head;
+
+    // copy page number i of this warp (tokens [16*(warp+4i), +16) of the chunk) into ring slot i % kStages
+    auto issue_page = [&](int i) {
+        if (i < my_pages) {
+            const int page_in_chunk = warp + i * kWarps;
+            const int64_t page = __ldg(my_page_ids + page_in_chunk);
+            const int valid = min(kPageSize, n_tok - page_in_chunk * kPageSize);
+            const uint32_t dst = warp_smem + (i % kStages) * L::kStageBytes;
+            const __nv_bfloat16 *src_k = head_k + page * stride_page;
+            const __nv_bfloat16 *src_v = head_v + page * stride_page;
+#pragma unroll
+            for (int c = lane; c < kPageSize * CPR; c += 32) {
+                const int row = c / CPR, col = c % CPR;
+                const int bytes = row < valid ? 16 : 0;              // 0: nothing is read, the slot is zero-filled
+                const int64_t off = bytes ? row * stride_tok + col * 8 : 0;
+                const uint32_t d = dst + row * L::kRowBytes + ((col ^ (row & 7)) << 4);
+                cp_async16(d, src_k + off, bytes);
+                cp_async16(d + L::kPageBytes, src_v + off, bytes);
+            }
+        }
+        cp_async_commit();  // an empty group keeps the group count uniform
+    };
+
+    float o[DN][4];
+#pragma unroll
+    for (int n = 0; n < DN; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+    float m_ref = -INFINITY;  // reference maximum of row qrow, in log2 units (uniform over the quad)
+    float l_part = 0.f;       // this thread's share of the row sum
+
+#pragma unroll
+    for (int i = 0; i < kStages - 1; ++i) issue_page(i);
+
+    for (int i = 0; i < my_pages; ++i) {
+        cp_async_wait<kStages - 2>();
+        __syncwarp();
+        issue_page(i + kStages - 1);  // refills the slot read in iteration i - 1
+
+        const int page_in_chunk = warp + i * kWarps;
+        const int valid = min(kPageSize, n_tok - page_in_chunk * kPageSize);
+        const uint32_t sk = warp_smem + (i % kStages) * L::kStageBytes;
+        const uint32_t sv = sk + L::kPageBytes;
+
+        // ---- S = Q K^T for 16 tokens: two 16x8 accumulators
+        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        {
+            const int mat = lane >> 3, r = lane & 7;
+            const int tok = (mat >> 1) * 8 + r;
+            const uint32_t row_addr = sk + tok * L::kRowBytes;
+#pragma unroll
+            for (int kk = 0; kk < KK; ++kk) {
+                const int chunk = 2 * kk + (mat & 1);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4(row_addr + ((chunk ^ (tok & 7)) << 4), b0, b1, b2, b3);
+                mma_bf16(sc[0], qa0[kk], 0u, qa2[kk], 0u, b0, b1);
+                mma_bf16(sc[1], qa0[kk], 0u, qa2[kk], 0u, b2, b3);
+            }
+        }
+        // this thread holds row qrow, tokens {qcol, qcol+1, 8+qcol, 8+qcol+1}
+        float x[4];
+        x[0] = sc[0][0] * scale_log2; x[1] = sc[0][1] * scale_log2;
+        x[2] = sc[1][0] * scale_log2; x[3] = sc[1][1] * scale_log2;
+        if (valid < kPageSize) {
+            if (qcol >= valid) x[0] = -INFINITY;
+            if (qcol + 1 >= valid) x[1] = -INFINITY;
+            if (qcol + 8 >= valid) x[2] = -INFINITY;
+            if (qcol + 9 >= valid) x[3] = -INFINITY;
+        }
+        const float tmax = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+        if (__any_sync(0xffffffffu, tmax > m_ref + kRescaleThreshold)) {
+            float rmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+            rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 2));
+            const float m_new = fmaxf(m_ref, rmax);
+            if (m_new > m_ref) {  // quad-uniform
+                const float alpha = fast_exp2(m_ref - m_new);  // m_ref = -inf gives 0
+                l_part *= alpha;
+#pragma unroll
+                for (int n = 0; n < DN; ++n) { o[n][0] *= alpha; o[n][1] *= alpha; }
+                m_ref = m_new;
+            }
+        }
+        float p[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) p[t] = fast_exp2(x[t] - m_ref);  // masked slots: exp2(-inf) = 0
+        l_part += (p[0] + p[1]) + (p[2] + p[3]);
+        const uint32_t pa0 = pack_bf16(p[0], p[1]), pa2 = pack_bf16(p[2], p[3]);
+
+        // ---- O += P V : V[16 tokens x D] read transposed, two 8-wide column tiles per ldmatrix
+        {
+            const int mat = lane >> 3, r = lane & 7;
+            const int tok = (mat & 1) * 8 + r;
+            const uint32_t row_addr = sv + tok * L::kRowBytes;
+#pragma unroll
+            for (int n = 0; n < DN; n += 2) {
+                const int chunk = n + (mat >> 1);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(row_addr + ((chunk ^ (tok & 7)) << 4), b0, b1, b2, b3);
+                mma_bf16(o[n], pa0, 0u, pa2, 0u, b0, b1);
+                mma_bf16(o[n + 1], pa0, 0u, pa2, 0u, b2, b3);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- finish the row sum inside the quad, then combine the 4 warps through shared memory
+    float l_row = l_part + __shfl_xor_sync(0xffffffffu, l_part, 1);
+    l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
+    __syncthreads();  // every warp is done with its ring: reuse the memory
+    float *sm_o = reinterpret_cast<float *>(smem_raw);           // [kWarps][G][D]
+    float *sm_m = sm_o + kWarps * G * D;                          // [kWarps][G]
+    float *sm_l = sm_m + kWarps * G;                              // [kWarps][G]
+    if (qrow < G) {
+        float *dst = sm_o + (warp * G + qrow) * D + qcol;
+#pragma unroll
+        for (int n = 0; n < DN; ++n) *reinterpret_cast<float2 *>(dst + n * 8) = make_float2(o[n][0], o[n][1]);
+        if ((lane & 3) == 0) { sm_m[warp * G + qrow] = m_ref; sm_l[warp * G + qrow] = l_row; }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < G * D; e += kWarps * 32) {
+        const int g = e / D, d = e % D;
+        float top = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) top = fmaxf(top, sm_m[w * G + g]);
+        float z = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float mw = sm_m[w * G + g];
+            const float f = mw == -INFINITY ? 0.f : fast_exp2(mw - top);
+            z += f * sm_l[w * G + g];
+            acc += f * sm_o[(w * G + g) * D + d];
+        }
+        partial_o[size_t(prow0 + g) * D + d] = acc / z;
+        if (d == 0) partial_lse[prow0 + g] = (top + log2f(z)) * 0.6931471805599453f;
+    }
+}
+
+template <int D, int G>
+int launch_one(const SuffixArgs &a, cudaStream_t st)
+{
+    using L = SuffixSmem<D>;
+    static_assert(L::kTotal >= int(sizeof(float)) * kWarps * G * (D + 2), "combine buffer must fit in the ring");
+    auto kern = suffix_kernel<D, G>;
+    static bool configured = false;  // attribute set once per process and instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return int(e);
+        configured = true;
+    }
+    const float scale_log2 = a.sm_scale * 1.4426950408889634f;
+    kern<<<a.num_items, kWarps * 32, L::kTotal, st>>>(
+        static_cast<const __nv_bfloat16 *>(a.q), static_cast<const __nv_bfloat16 *>(a.pool_k),
+        static_cast<const __nv_bfloat16 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok, a.page_indptr,
+        a.page_indices, a.suffix_lens, a.items, a.sample_info, a.num_q_heads, a.chunk_tokens, scale_log2, a.partial_o,
+        a.partial_lse);
+    return int(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_suffix(const SuffixArgs &a, void *stream, std::string *err)
+{
+    if (a.num_items == 0) return 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int G = a.num_q_heads / a.num_kv_heads;
+    int rc = -1;
+#define PSA_CASE(DD, GG) if (a.head_dim == DD && G == GG) rc = launch_one<DD, GG>(a, st);
+    PSA_CASE(128, 1) PSA_CASE(128, 2) PSA_CASE(128, 4) PSA_CASE(128, 8)
+    PSA_CASE(64, 1) PSA_CASE(64, 2) PSA_CASE(64, 4) PSA_CASE(64, 8)
+#undef PSA_CASE
+    if (rc != 0 && err) *err = rc < 0 ? "suffix: unsupported shape" : std::string("suffix launch: ") + cudaGetErrorString(cudaError_t(rc));
+    return rc;
+}
+
+}  // namespace psa

@@ -1,0 +1,287 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU fp64 oracle, element by element,
+on the same seeded inputs.  Tolerances: max |err| <= 1e-2 on out, <= 1e-3 on lse (absolute)."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import psa_workloads as wl
+from psa_testlib import assert_close, make_plan, run_gpu, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def cfg(**kw):
+    base = dict(name="t", num_prefixes=1, samples_per_prefix=4, num_q_heads=8, num_kv_heads=2, head_dim=128,
+                prefix_len=(300, 300), suffix_len=(0, 200), page_size=16, seed=11)
+    base.update(kw)
+    return wl.PsaConfig(**base)
+
+
+def check(w, out_dtype="bf16", rows=None, what="", **plan_kw):
+    plan = make_plan(w, out_dtype, **plan_kw) if plan_kw else None
+    out, lse, plan = run_gpu(w, out_dtype, plan=plan)
+    if rows is None:
+        ref_o, ref_l, _ = oracle.attend(w)
+    else:
+        ref_o, ref_l, _ = oracle.attend(w, rows=rows)
+        out, lse = out[rows], lse[rows]
+    return assert_close(out, lse, ref_o, ref_l, what)
+
+
+# ------------------------------------------------------------------ the named configurations
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3"])
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_named_config_every_element(name, out_dtype):
+    w = wl.make_workload(wl.CONFIGS[name], poison=True)
+    check(w, out_dtype, what=f"{name}/{out_dtype}")
+
+
+@pytest.mark.parametrize("name", ["cfg4", "cfg5"])
+def test_full_size_config_sampled_rows(name):
+    """Full size, the launch configuration the benchmark times; the oracle computes a sample of the
+    rows one by one: rows of the shortest and longest suffixes plus 192 random rows.  Everything
+    else is checked for being finite and bounded by the value range."""
+    w = wl.make_workload(wl.CONFIGS[name], poison=True)
+    Hq = w["num_q_heads"]
+    S = w["suffix_lens"]
+    rng = np.random.default_rng(123)
+    pick = set(rng.choice(len(S) * Hq, 192, replace=False).tolist())
+    for s in (int(np.argmin(S)), int(np.argmax(S))):
+        pick.update(range(s * Hq, (s + 1) * Hq))
+    rows = np.array(sorted(pick), dtype=np.int64)
+    out, lse, plan = run_gpu(w, "bf16")
+    ref_o, ref_l, _ = oracle.attend(w, rows=rows)
+    assert_close(out[rows], lse[rows], ref_o, ref_l, name)
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+    vmax = float(np.max(np.abs(wl.bf16_bits_to_f32(w["prefix_v"][:4096]))))
+    assert np.max(np.abs(out)) <= max(vmax, 6.0)        # a convex combination of N(0,1) values
+
+
+# ------------------------------------------------------------------ shapes around every tile / page edge
+@pytest.mark.parametrize("D,G", [(128, 4), (128, 8), (128, 1), (128, 2), (64, 4), (64, 8), (64, 1), (64, 2)])
+def test_head_dim_and_group_sizes(D, G):
+    w = wl.make_workload(cfg(head_dim=D, num_q_heads=2 * G, num_kv_heads=2, samples_per_prefix=5,
+                             prefix_len=(333, 333), suffix_len=(0, 150)), poison=True)
+    check(w, "f32", what=f"D{D} G{G}")
+
+
+@pytest.mark.parametrize("L", [0, 1, 15, 127, 128, 129, 255, 256, 257, 1000])
+def test_prefix_lengths_around_tile_edges(L):
+    w = wl.make_workload(cfg(prefix_len=(L, L), suffix_len=(1, 40)), poison=True)
+    check(w, "f32", what=f"L{L}")
+
+
+def test_suffix_lengths_around_page_and_chunk_edges():
+    lens = [0, 1, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 511, 513, 1023, 1025]
+    c = cfg(samples_per_prefix=len(lens), prefix_len=(64, 64))
+    w = wl.make_workload(c, poison=True, lengths=([64], [len(lens)], lens))
+    check(w, "f32", what="suffix edges")
+    check(w, "bf16", what="suffix edges bf16")
+
+
+@pytest.mark.parametrize("n_samples", [1, 31, 32, 33, 63, 64, 65, 70])
+def test_row_counts_around_row_tile_edges(n_samples):
+    # G = 4: 32 samples fill one 128-row tile, 64 fill the 256 rows of one item
+    w = wl.make_workload(cfg(samples_per_prefix=n_samples, num_q_heads=4, num_kv_heads=1,
+                             prefix_len=(200, 200), suffix_len=(0, 20)), poison=True)
+    check(w, "f32", what=f"N{n_samples}")
+
+
+def test_many_prompts_ragged_everything():
+    rng = np.random.default_rng(4)
+    P = 7
+    prefix_lens = [0, 1, 130, 777, 128, 2049, 300]
+    n_samples = [3, 0, 40, 2, 70, 1, 5]
+    B = sum(n_samples)
+    suffix_lens = rng.integers(0, 300, size=B)
+    suffix_lens[:3] = 0                      # prompt 0 has no prefix: those rows have an empty context
+    w = wl.make_workload(cfg(num_prefixes=P, permute_pages=True), poison=True,
+                         lengths=(prefix_lens, n_samples, suffix_lens))
+    eo, el = check(w, "f32", what="ragged")
+    out, lse, _ = run_gpu(w, "bf16")
+    assert (lse[: 3 * 8] == -math.inf).all() and (out[: 3 * 8] == 0).all()
+
+
+def test_all_contexts_empty():
+    w = wl.make_workload(cfg(prefix_len=(0, 0), suffix_len=(0, 0)))
+    out, lse, _ = run_gpu(w, "bf16")
+    assert (out == 0).all() and (lse == -math.inf).all()
+
+
+def test_multi_split_prefix_and_multi_chunk_suffix_small_sm_count():
+    # planning for few SMs and for many SMs must give the same numbers
+    w = wl.make_workload(cfg(prefix_len=(3000, 3000), suffix_len=(100, 900), samples_per_prefix=6), poison=True)
+    for sms in (1, 4, 148, 1000):
+        check(w, "f32", what=f"sms{sms}", num_sms=sms)
+
+
+# ------------------------------------------------------------------ layouts, plan reuse
+def test_strided_layouts_head_major_prefix_and_token_major_pool():
+    import torch
+    from paper_2502_02534_b200 import decode
+    w = wl.make_workload(cfg(), poison=True)
+    ref_o, ref_l, _ = oracle.attend(w)
+    dev = to_device(w)
+    Hkv, D, page = w["num_kv_heads"], w["head_dim"], w["page_size"]
+    L = w["prefix_k"].shape[0]
+    pk = dev["prefix_k"].permute(1, 0, 2).contiguous()      # [Hkv, L, D]
+    pv = dev["prefix_v"].permute(1, 0, 2).contiguous()
+    sk = dev["pool_k"].permute(0, 2, 1, 3).contiguous()     # [pages, 16, Hkv, D]
+    sv = dev["pool_v"].permute(0, 2, 1, 3).contiguous()
+    plan = make_plan(w, "f32")
+    B, Hq = int(np.sum(w["n_samples"])), w["num_q_heads"]
+    out = torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+    decode(plan, dev["q"], pk, pv, sk, sv, dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], out, lse,
+           prefix_strides=(D, L * D), pool_strides=(page * Hkv * D, D, Hkv * D))
+    torch.cuda.synchronize()
+    plan.check_status()
+    assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, "strided")
+
+
+def test_plan_reuse_with_shorter_actual_suffixes_and_growth():
+    """A plan made for upper bounds serves every step whose lengths stay below them."""
+    c = cfg(samples_per_prefix=6, suffix_len=(50, 400))
+    w = wl.make_workload(c, poison=False)
+    bounds = np.asarray(w["suffix_lens"]).copy()
+    plan = make_plan(w, "f32", suffix_bounds=bounds)
+    dev = to_device(w)
+    import torch
+    for shrink in (0, 1, 17, 49):
+        w2 = dict(w)
+        w2["suffix_lens"] = np.maximum(bounds - shrink, 0).astype(np.int32)
+        dev["suffix_lens"] = torch.from_numpy(w2["suffix_lens"]).cuda()
+        out, lse, _ = run_gpu(w2, "f32", plan=plan, dev=dev)
+        ref_o, ref_l, _ = oracle.attend(w2)
+        assert_close(out, lse, ref_o, ref_l, f"shrink{shrink}")
+
+
+# ------------------------------------------------------------------ adversarial values
+def test_late_large_logit_forces_accumulator_rescale():
+    """A key far into the context with a logit ~40 above everything before it: the running maximum
+    must move and the accumulated output must be rescaled (prefix in TMEM, suffix in registers)."""
+    c = cfg(samples_per_prefix=3, prefix_len=(700, 700), suffix_len=(90, 90), num_q_heads=4, num_kv_heads=1)
+    w = wl.make_workload(c, poison=True)
+    D = w["head_dim"]
+    q0 = wl.bf16_bits_to_f32(w["q"][0, 0])
+    big = wl.f32_to_bf16_bits(q0 * (40.0 / (w["sm_scale"] * float(q0 @ q0))))
+    w["prefix_k"][650, 0] = big                # tile 5 of the prefix
+    pg = w["page_indices"][w["page_indptr"][1] + 80 // 16]
+    q1 = wl.bf16_bits_to_f32(w["q"][1, 1])
+    w["pool_k"][pg, 0, 80 % 16] = wl.f32_to_bf16_bits(q1 * (60.0 / (w["sm_scale"] * float(q1 @ q1))))
+    ref_o, ref_l, _ = oracle.attend(w)
+    assert ref_l[0] > 35 and ref_l[1 * 4 + 1] > 55
+    out, lse, _ = run_gpu(w, "f32")
+    assert_close(out, lse, ref_o, ref_l, "rescale")
+
+
+def test_all_keys_equal_closed_form():
+    c = cfg(samples_per_prefix=2, prefix_len=(257, 257), suffix_len=(33, 33), num_q_heads=4, num_kv_heads=1)
+    w = wl.make_workload(c, poison=True)
+    k = w["prefix_k"][0, 0].copy()
+    w["prefix_k"][:] = k
+    pk = w["pool_k"]
+    pk[pk != wl.BF16_NAN] = 0
+    for pg in w["page_indices"]:
+        n = w["pool_k"][pg, 0].shape[0]
+        for t in range(n):
+            if w["pool_k"][pg, 0, t, 0] != wl.BF16_NAN:
+                w["pool_k"][pg, 0, t] = k
+    out, lse, _ = run_gpu(w, "f32")
+    q = wl.bf16_bits_to_f32(w["q"]).astype(np.float64).reshape(-1, 128)
+    x = w["sm_scale"] * (q @ wl.bf16_bits_to_f32(k).astype(np.float64))
+    assert np.max(np.abs(lse - (x + math.log(257 + 33)))) <= 1e-3
+    ref_o, ref_l, _ = oracle.attend(w)
+    assert_close(out, lse, ref_o, ref_l, "equal keys")
+
+
+def test_permuting_samples_permutes_rows_only():
+    c = cfg(samples_per_prefix=8, permute_pages=True)
+    w = wl.make_workload(c, poison=True)
+    out, lse, _ = run_gpu(w, "f32")
+    perm = np.array([5, 2, 7, 0, 3, 6, 1, 4])
+    B, Hq, D = 8, w["num_q_heads"], w["head_dim"]
+    w2 = dict(w)
+    w2["q"] = w["q"][perm]; w2["suffix_lens"] = w["suffix_lens"][perm]
+    lists = [w["page_indices"][w["page_indptr"][s]: w["page_indptr"][s + 1]] for s in range(B)]
+    w2["page_indices"] = np.concatenate([lists[s] for s in perm]).astype(np.int32)
+    w2["page_indptr"] = np.concatenate([[0], np.cumsum([len(lists[s]) for s in perm])]).astype(np.int32)
+    o2, l2, _ = run_gpu(w2, "f32")
+    # the work lists differ (chunks are ordered by length), so equality is up to summation order
+    assert np.max(np.abs(o2.reshape(B, Hq, D) - out.reshape(B, Hq, D)[perm])) <= 1e-5
+    assert np.max(np.abs(l2.reshape(B, Hq) - lse.reshape(B, Hq)[perm])) <= 1e-5
+
+
+# ------------------------------------------------------------------ stages and the host-buffer entry point
+def test_stage_entry_points_compose_to_decode():
+    import torch
+    from paper_2502_02534_b200 import decode
+    w = wl.make_workload(cfg(), poison=True)
+    dev = to_device(w)
+    plan = make_plan(w, "f32")
+    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    out = torch.zeros((B, Hq, D), dtype=torch.float32, device="cuda"); lse = torch.zeros((B, Hq), dtype=torch.float32, device="cuda")
+    args = (plan, dev["q"], dev["prefix_k"], dev["prefix_v"], dev["pool_k"], dev["pool_v"], dev["page_indptr"],
+            dev["page_indices"], dev["suffix_lens"], out, lse)
+    for stage in ("suffix", "prefix", "merge"):
+        decode(*args, stage=stage)
+    torch.cuda.synchronize()
+    ref_o, ref_l, _ = oracle.attend(w)
+    assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, "stages")
+
+
+def test_decode_from_host_buffers():
+    import torch
+    from paper_2502_02534_b200 import decode_host
+    from paper_2502_02534_b200.binding import host_staging_bytes
+    w = wl.make_workload(wl.CONFIGS["cfg1"], poison=True)
+    plan = make_plan(w, "bf16")
+    plan.bind_workspace()
+    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    nbytes = host_staging_bytes(plan, w["prefix_k"].shape[0], w["pool_k"].shape[0], len(w["page_indices"]))
+    staging = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, Hq, D), dtype=torch.bfloat16).pin_memory(); lse = torch.empty((B, Hq), dtype=torch.float32).pin_memory()
+    i32 = lambda a: np.ascontiguousarray(a, dtype=np.int32)
+    decode_host(plan, w["q"], w["prefix_k"], w["prefix_v"], w["pool_k"], w["pool_v"], i32(w["page_indptr"]),
+                i32(w["page_indices"]), i32(w["suffix_lens"]), out, lse, staging)
+    torch.cuda.synchronize()
+    plan.check_status()
+    ref_o, ref_l, _ = oracle.attend(w)
+    assert_close(out.float().double().numpy().reshape(B * Hq, D), lse.double().numpy().reshape(-1), ref_o, ref_l, "host")
+
+
+def test_misuse_returns_status_codes_not_faults():
+    import torch
+    from paper_2502_02534_b200 import PsaError, decode
+    w = wl.make_workload(cfg())
+    dev = to_device(w)
+    plan = make_plan(w)
+    plan.bind_workspace()
+    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    out = torch.zeros((B, Hq, D), dtype=torch.bfloat16, device="cuda"); lse = torch.zeros((B, Hq), dtype=torch.float32, device="cuda")
+    good = [plan, dev["q"], dev["prefix_k"], dev["prefix_v"], dev["pool_k"], dev["pool_v"], dev["page_indptr"],
+            dev["page_indices"], dev["suffix_lens"], out, lse]
+    for idx in (1, 2, 4, 6, 9, 10):                    # a null pointer in each position
+        bad = list(good); bad[idx] = None
+        with pytest.raises(PsaError) as e:
+            decode(*bad)
+        assert e.value.status == 1
+    with pytest.raises(PsaError) as e:                 # misaligned q
+        bad = list(good); bad[1] = dev["q"].view(-1)[1:]
+        decode(*bad)
+    assert e.value.status == 1
+    with pytest.raises(PsaError) as e:                 # stride not a multiple of 8 elements
+        decode(*good, prefix_strides=(Hq * D + 1, D))
+    assert e.value.status == 1
+    small = plan.workspace[: plan.workspace_bytes - 256]
+    keep = plan.workspace
+    plan.workspace = small
+    with pytest.raises(PsaError) as e:
+        decode(*good)
+    assert e.value.status == 3
+    plan.workspace = keep
+    decode(*good)                                      # and the context is still healthy
+    torch.cuda.synchronize()
+    plan.check_status()
