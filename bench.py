@@ -1,0 +1,314 @@
+#!/usr/bin/env python
+"""Benchmark of one decode step of parallel-sample shared-prefix attention on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg2] [--impl psa|reference]
+
+A step = prefix + suffix + merge stages over one batch of seeded synthetic inputs (the shapes of
+the paper's parallel-sampling set-up; nothing is read from disk).  Rank r works on its own
+prompts (seed r): the path shards over independent prompts with no collective ("weak" scaling).
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import psa_workloads as wl  # noqa: E402
+
+METRIC = "sample-tokens/sec per decode step"
+UNIT = "sample-tokens/s"
+L2_BYTES = 126e6
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while work runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---------------------------------------------------------------------------------------------- reference arm
+def run_reference(args, cfg):
+    """The CPU fp64 oracle as it stands, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    w = wl.make_workload(cfg)
+    B, Hq = int(np.sum(w["n_samples"])), w["num_q_heads"]
+    n_rows = B * Hq
+    t0 = time.perf_counter()
+    oracle.attend(w)
+    t_full = time.perf_counter() - t0
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    if t_full <= budget:
+        rows, sample = None, f"every row of {cfg.name} ({n_rows} rows) per step"
+        rows_per_step = n_rows
+    else:
+        rows_per_step = max(Hq, int(n_rows * budget / t_full) // Hq * Hq)
+        sel = np.random.default_rng(0).choice(B, rows_per_step // Hq, replace=False)
+        rows = (np.sort(sel)[:, None] * Hq + np.arange(Hq)[None, :]).ravel()
+        sample = f"{rows_per_step // Hq} of {B} samples of {cfg.name} (all {Hq} heads) per step"
+    cores = 0
+    for _ in range(args.warmup):
+        oracle.attend(w, rows=rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        _, _, cores = oracle.attend(w, rows=rows)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = (rows_per_step / Hq) / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": cfg.name, "note": "CPU fp64 oracle on host cores"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- psa arm
+def run_psa(args, cfg):
+    import torch
+    import torch.distributed as dist
+    import paper_2502_02534_b200 as psa
+    from paper_2502_02534_b200.binding import host_staging_bytes
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- inputs: rank r samples its own prompts (seed r); several copies so no step finds its inputs in L2
+    import dataclasses
+    cfg_r = dataclasses.replace(cfg, seed=cfg.seed + rank)
+    w = wl.make_workload(cfg_r)
+    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    abytes, aflops = wl.algorithmic_bytes(w), wl.algorithmic_flops(w)
+    input_bytes = sum(int(w[k].nbytes) for k in ("q", "prefix_k", "prefix_v", "pool_k", "pool_v"))
+    n_copies = max(2, int(np.ceil(4 * L2_BYTES / input_bytes))) if input_bytes < 4 * L2_BYTES else 1
+
+    def upload():
+        d = {k: torch.from_numpy(np.ascontiguousarray(w[k]).view(np.int16)).cuda().view(torch.bfloat16)
+             for k in ("q", "prefix_k", "prefix_v", "pool_k", "pool_v")}
+        for k in ("page_indptr", "page_indices", "suffix_lens"):
+            d[k] = torch.from_numpy(np.ascontiguousarray(w[k], dtype=np.int32)).cuda()
+        return d
+
+    copies = [upload() for _ in range(n_copies)]
+    out = torch.empty((B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+    plan = psa.Plan(w["prefix_lens"], w["n_samples"], w["suffix_lens"], num_q_heads=Hq, num_kv_heads=w["num_kv_heads"],
+                    head_dim=D, page_size=w["page_size"], sm_scale=w["sm_scale"], out_dtype="bf16")
+    plan.bind_workspace()
+    info = plan.info
+
+    def step(i, stage="all"):
+        d = copies[i % n_copies]
+        psa.decode(plan, d["q"], d["prefix_k"], d["prefix_v"], d["pool_k"], d["pool_v"], d["page_indptr"],
+                   d["page_indices"], d["suffix_lens"], out, lse, stage=stage)
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    plan.check_status()
+
+    # ---- per-stage durations: same steps, same rotation, events around each stage
+    stage_ms = {"prefix": [], "suffix": [], "merge": []}
+    n_kt = min(args.steps, 200)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_kt)]
+    for i in range(n_kt):
+        evs[i][0].record(); step(i, "prefix")
+        evs[i][1].record(); step(i, "suffix")
+        evs[i][2].record(); step(i, "merge")
+        evs[i][3].record()
+    torch.cuda.synchronize()
+    for i in range(n_kt):
+        for j, name in enumerate(("prefix", "suffix", "merge")):
+            stage_ms[name].append(evs[i][j].elapsed_time(evs[i][j + 1]))
+    stage_avg = {k: (sum(v) / len(v) if v else None) for k, v in stage_ms.items()}
+
+    # ---- end to end through the host-buffer entry point: pinned host inputs, H2D + step + D2H every step
+    pin = {k: torch.from_numpy(np.ascontiguousarray(w[k]).view(np.int16)).pin_memory()
+           for k in ("q", "prefix_k", "prefix_v", "pool_k", "pool_v")}
+    for k in ("page_indptr", "page_indices", "suffix_lens"):
+        pin[k] = torch.from_numpy(np.ascontiguousarray(w[k], dtype=np.int32)).pin_memory()
+    out_h = torch.empty((B, Hq, D), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty((B, Hq), dtype=torch.float32).pin_memory()
+    n_tok, n_pages, n_idx = w["prefix_k"].shape[0], w["pool_k"].shape[0], len(w["page_indices"])
+    staging = torch.empty(host_staging_bytes(plan, n_tok, n_pages, n_idx), dtype=torch.uint8, device="cuda")
+    h2d = sum(int(pin[k].numel() * pin[k].element_size()) for k in pin)
+    d2h = int(out_h.numel() * 2 + lse_h.numel() * 4)
+
+    def e2e_step():
+        psa.decode_host(plan, pin["q"], pin["prefix_k"], pin["prefix_v"], pin["pool_k"], pin["pool_v"], pin["page_indptr"],
+                        pin["page_indices"], pin["suffix_lens"], out_h, lse_h, staging)
+
+    e2e_steps = max(1, min(args.steps, int(20.0 / max(1e-4, h2d / 20e9))))   # keep this leg to ~20 s at worst
+    for _ in range(min(3, args.warmup)):
+        e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
+    clocks = sampler.stop()
+
+    # ---- max over ranks
+    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(times[0]), float(times[1])
+    ms_step = ms_total / args.steps
+    value = world * B / (ms_step * 1e-3)
+
+    if rank == 0:
+        peaks, peaks_kind = load_peaks()
+        hbm = float(peaks["hbm_gbs"])
+        tf = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1400.0)))
+        suf_gbs = abytes["suffix"] / (stage_avg["suffix"] * 1e-3) / 1e9 if stage_avg["suffix"] else None
+        kernels = {}
+        for name in ("prefix", "suffix"):
+            t_roof_ms = max(abytes[name] / (hbm * 1e9), aflops[name] / (tf * 1e12)) * 1e3
+            kernels[name] = {"ms": stage_avg[name], "algorithmic_bytes": abytes[name], "flops": aflops[name],
+                             "t_roof_ms": t_roof_ms, "frac_of_roofline": t_roof_ms / stage_avg[name] if stage_avg[name] else None}
+        kernels["merge"] = {"ms": stage_avg["merge"]}
+        t_roof_step = max((abytes["prefix"] + abytes["suffix"]) / (hbm * 1e9), (aflops["prefix"] + aflops["suffix"]) / (tf * 1e12)) * 1e3
+        # CPU baseline: the oracle as it stands, on this machine's host cores, one full step of the same workload
+        import oracle
+        best, cores = None, 0
+        for _ in range(3):
+            t0 = time.perf_counter()
+            _, _, cores = oracle.attend(w)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "prompts": cfg.num_prefixes, "samples": B, "q_heads": Hq,
+                       "kv_heads": w["num_kv_heads"], "head_dim": D, "prefix_len": list(cfg.prefix_len),
+                       "suffix_len": list(cfg.suffix_len), "page_size": 16,
+                       "cold_l2": f"steps rotate over {n_copies} input copies ({n_copies * input_bytes / 1e6:.0f} MB > L2 126 MB)",
+                       "sharding": "independent prompts per rank, no collective"},
+            "plan": {"prefix_items": info.num_prefix_items, "suffix_items": info.num_suffix_items,
+                     "prefix_tiles_per_item": info.prefix_tiles_per_item, "suffix_chunk_tokens": info.suffix_chunk_tokens},
+            "gpu_launches": info.kernel_launches * args.steps,
+            "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps, "entry_point": "psa_decode_host"},
+            "roofline": {"kernel": "suffix_kernel", "bound": "hbm", "achieved": suf_gbs, "peak": hbm, "unit": "GB/s",
+                         "frac": suf_gbs / hbm if suf_gbs else None, "traffic": None, "peak_kind": f"of {peaks_kind}",
+                         "algorithmic_bytes_per_launch": abytes["suffix"]},
+            "kernels": kernels,
+            "step_roofline": {"t_roof_ms": t_roof_step, "frac": t_roof_step / ms_step},
+            "cpu_baseline": {"value": B / best, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"one full {cfg.name} step ({B * Hq} rows), best of 3"},
+            "clocks": clocks,
+            "input_checksum": wl.checksum(w),
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", default="cfg2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup) if args.impl == "psa" else args.warmup
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_psa(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
