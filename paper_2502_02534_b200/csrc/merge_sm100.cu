@@ -6,7 +6,8 @@
 //     lse = ln sum_i exp(lse_i),   out = sum_i exp(lse_i - lse) O_i .
 // A row with no partial at all (empty prefix and empty suffix) gives out = 0, lse = -inf.
 //
-// One warp per row; lane l owns D/32 consecutive output elements.  The stage moves
+// One warp per row; lane l owns D/32 consecutive output elements.  Partials are read with
+// L2-only loads (they were written by other blocks moments ago).  The stage moves
 // (#partials * D * 4 + D * 2) bytes per row and is bound by L2 / HBM bandwidth.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -16,7 +17,7 @@
 namespace psa {
 namespace {
 
-constexpr int kMergeWarps = 8;
+constexpr int kMergeWarps = 4;
 
 template <int D>
 __global__ void __launch_bounds__(kMergeWarps * 32)
@@ -49,28 +50,51 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
 
     // pass 1: the largest lse (lanes stride over the partials)
     float top = -INFINITY;
-    for (int i = lane; i < n_total; i += 32) top = fmaxf(top, __ldg(partial_lse + partial_row(i)));
+    for (int i = lane; i < n_total; i += 32) top = fmaxf(top, __ldcg(partial_lse + partial_row(i)));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, o));
 
+    // pass 2: lane i of each group of 32 partials computes weight and row; the rows are then
+    // fetched four at a time so that several loads are in flight per lane
     float acc[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = 0.f;
     float z = 0.f;
+    auto fetch = [&](int r) {
+        const float *src = partial_o + size_t(r) * D + lane * V;
+        if constexpr (V == 4) return __ldcg(reinterpret_cast<const float4 *>(src));
+        else { const float2 x = __ldcg(reinterpret_cast<const float2 *>(src)); return make_float4(x.x, x.y, 0.f, 0.f); }
+    };
+    auto fma_row = [&](float w, const float4 &x) {
+        acc[0] += w * x.x; acc[1] += w * x.y;
+        if constexpr (V == 4) { acc[2] += w * x.z; acc[3] += w * x.w; }
+    };
     if (top != -INFINITY) {
-        for (int i = 0; i < n_total; ++i) {
-            const int r = partial_row(i);
-            const float w = __expf(__ldg(partial_lse + r) - top);  // 0 for an empty piece (lse = -inf)
-            z += w;
-            const float *src = partial_o + size_t(r) * D + lane * V;
-            if constexpr (V == 4) {
-                const float4 x = __ldg(reinterpret_cast<const float4 *>(src));
-                acc[0] += w * x.x; acc[1] += w * x.y; acc[2] += w * x.z; acc[3] += w * x.w;
-            } else {
-                const float2 x = __ldg(reinterpret_cast<const float2 *>(src));
-                acc[0] += w * x.x; acc[1] += w * x.y;
+        for (int base = 0; base < n_total; base += 32) {
+            const int mine = base + lane;
+            const int my_row = mine < n_total ? partial_row(mine) : 0;
+            // an empty piece (lse = -inf) gets weight 0
+            const float my_w = mine < n_total ? __expf(__ldcg(partial_lse + my_row) - top) : 0.f;
+            z += my_w;
+            const int cnt = min(32, n_total - base);
+            int i = 0;
+            for (; i + 4 <= cnt; i += 4) {
+                float4 x[4]; float w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    w[u] = __shfl_sync(0xffffffffu, my_w, i + u);
+                    x[u] = fetch(__shfl_sync(0xffffffffu, my_row, i + u));
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) fma_row(w[u], x[u]);
+            }
+            for (; i < cnt; ++i) {
+                const float w = __shfl_sync(0xffffffffu, my_w, i);
+                fma_row(w, fetch(__shfl_sync(0xffffffffu, my_row, i)));
             }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
         const float inv = 1.f / z;
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] *= inv;
