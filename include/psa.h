@@ -146,6 +146,38 @@ psa_status_t psa_decode(const psa_plan_t *plan, const void *q,
                         void *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * psa_decode without a caller workspace and without any allocation.  (The paper has no
+ * counterpart for this entry point; it exists for how the library gets embedded.)
+ *
+ * Who needs it: callers that are not allowed to allocate device memory around a decode step --
+ * a plugin inside a serving process whose memory pool already owns the whole GPU, code
+ * running under an allocator it does not control, or a latency-critical loop in which a
+ * cudaMalloc would stall the device.  The scratch memory of the step (work lists, status
+ * word, partial results of the prefix and suffix stages) lives in one fixed array of
+ * PSA_STATIC_WORKSPACE_BYTES inside the library image; every GPU that loads the library
+ * holds that much memory until the process ends.  This function calls no cudaMalloc,
+ * cudaFree or other allocating routine; it copies the plan's work lists into the array
+ * (which also clears the status word) and then runs the same three stages as psa_decode,
+ * on `cuda_stream`, without synchronising.  All other arguments are those of psa_decode.
+ *
+ *   - A plan whose psa_plan_workspace_bytes exceeds PSA_STATIC_WORKSPACE_BYTES is rejected
+ *     with PSA_ERR_WORKSPACE (the message names both sizes); nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps what the last call left in
+ *     it.  Two calls whose GPU work can overlap (different streams, different threads or
+ *     different plans) race on it: serialise them, or give one of them psa_decode with its
+ *     own workspace.  Device-side status of a step is not retrievable through
+ *     psa_check_status here; use psa_decode when that is needed.
+ */
+#define PSA_STATIC_WORKSPACE_BYTES (16u << 20)
+psa_status_t psa_decode_static(const psa_plan_t *plan, const void *q,
+                               const void *prefix_k, const void *prefix_v, const int64_t prefix_strides[2],
+                               const void *suffix_k_pool, const void *suffix_v_pool, const int64_t pool_strides[3],
+                               const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
+                               void *out, float *lse, void *cuda_stream);
+
+/*
  * The stages one by one, for tests and per-kernel timing.  Same arguments as psa_decode.
  * prefix and suffix write partial results into the workspace; merge reads them.
  */

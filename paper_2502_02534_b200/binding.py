@@ -17,7 +17,7 @@ PSA_OUT_BF16, PSA_OUT_F32 = 0, 1
 EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
-    "psa_decode", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
+    "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
     "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
@@ -81,6 +81,8 @@ def library():
         lib.psa_plan_suffix_items.argtypes = [P, P]
         lib.psa_decode.restype = c_int32
         lib.psa_decode.argtypes = [P, P, P, P, POINTER(c_int64), P, P, POINTER(c_int64), P, P, P, P, P, P, c_size_t, P]
+        lib.psa_decode_static.restype = c_int32
+        lib.psa_decode_static.argtypes = [P, P, P, P, POINTER(c_int64), P, P, POINTER(c_int64), P, P, P, P, P, P]
         lib.psa_decode_prefix.restype = c_int32
         lib.psa_decode_prefix.argtypes = [P, P, P, P, POINTER(c_int64), P, c_size_t, P]
         lib.psa_decode_suffix.restype = c_int32
@@ -229,6 +231,21 @@ def decode(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page
         _check(lib.psa_decode_merge(plan.handle, _ptr(suffix_lens), _ptr(out), _ptr(lse), ws, wsb, st))
     else:
         raise ValueError(stage)
+
+
+STATIC_WORKSPACE_BYTES = 16 << 20
+
+
+def decode_static(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices,
+                  suffix_lens, out, lse, *, prefix_strides=None, pool_strides=None, stream=None):
+    """psa_decode_static: the same step with the library's built-in scratch array instead of a
+    workspace tensor -- nothing is allocated, here or in the library.  Calls that may overlap on
+    the GPU share that array and must be serialised by the caller."""
+    pst = _strides(prefix_strides or default_prefix_strides(plan), 2)
+    qst = _strides(pool_strides or default_pool_strides(plan), 3)
+    _check(library().psa_decode_static(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, _ptr(suffix_k_pool),
+                                       _ptr(suffix_v_pool), qst, _ptr(page_indptr), _ptr(page_indices),
+                                       _ptr(suffix_lens), _ptr(out), _ptr(lse), _stream_ptr(stream)))
 
 
 def decode_host(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,

@@ -48,6 +48,10 @@ psa_status_t carve(const psa_plan_t *plan, void *workspace, size_t bytes, Carved
 
 }  // namespace
 
+namespace psa {
+psa_status_t set_last_error(psa_status_t status, const std::string &message) { return fail(status, message); }
+}  // namespace psa
+
 extern "C" {
 
 psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes, const int32_t *prefix_lens,

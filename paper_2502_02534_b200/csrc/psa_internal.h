@@ -86,6 +86,9 @@ struct psa_plan {
 
 namespace psa {
 
+// api.cu: records the thread-local message psa_last_error_message returns; returns `status`
+psa_status_t set_last_error(psa_status_t status, const std::string &message);
+
 // plan.cpp
 psa_status_t build_plan(const psa_config_t &cfg, int32_t num_prefixes, const int32_t *prefix_lens,
                         const int32_t *n_samples, const int32_t *suffix_lens, psa_plan *plan, std::string *err);
