@@ -68,6 +68,8 @@ typedef struct {
     float   sm_scale;   /* multiplies q.k before the softmax; > 0 */
     int32_t out_dtype;  /* PSA_OUT_BF16 or PSA_OUT_F32 */
     int32_t num_sms;    /* SMs to plan for; 0 = ask the current CUDA device */
+    int32_t suffix_chunk_tokens;   /* tokens per suffix work item: 0 = planner's choice, else a multiple of 64 */
+    int32_t prefix_tiles_per_item; /* 128-key tiles per prefix work item: 0 = planner's choice */
     int32_t reserved;   /* must be 0 */
 } psa_config_t;
 

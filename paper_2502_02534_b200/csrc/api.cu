@@ -150,15 +150,17 @@ psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void
     a.num_q_heads = plan->cfg.num_q_heads; a.num_kv_heads = plan->cfg.num_kv_heads; a.head_dim = plan->cfg.head_dim;
     a.sm_scale = plan->cfg.sm_scale;
     a.items = c.prefix_items; a.num_items = int32_t(plan->prefix_items.size());
+    a.max_rows_per_item = plan->prefix_max_rows_per_item; a.max_tiles_per_item = plan->prefix_tiles_per_item;
     a.partial_o = c.partial_o; a.partial_lse = c.partial_lse; a.status = c.status;
     std::string err;
     if (psa::launch_prefix(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
     return PSA_OK;
 }
 
-psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void *suffix_k_pool, const void *suffix_v_pool,
-                               const int64_t pool_strides[3], const int32_t *page_indptr, const int32_t *page_indices,
-                               const int32_t *suffix_lens, void *workspace, size_t workspace_bytes, void *cuda_stream)
+static psa_status_t suffix_impl(const psa_plan_t *plan, const void *q, const void *suffix_k_pool, const void *suffix_v_pool,
+                                const int64_t pool_strides[3], const int32_t *page_indptr, const int32_t *page_indices,
+                                const int32_t *suffix_lens, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                                bool after_prefix)
 {
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
@@ -179,13 +181,22 @@ psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void
     a.items = c.suffix_items; a.sample_info = c.sample_info;
     a.num_items = int32_t(plan->suffix_items.size()); a.chunk_tokens = plan->suffix_chunk_tokens;
     a.partial_o = c.partial_o; a.partial_lse = c.partial_lse; a.status = c.status;
+    a.after_prefix = after_prefix;
     std::string err;
     if (psa::launch_suffix(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
     return PSA_OK;
 }
 
-psa_status_t psa_decode_merge(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse, void *workspace,
-                              size_t workspace_bytes, void *cuda_stream)
+psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void *suffix_k_pool, const void *suffix_v_pool,
+                               const int64_t pool_strides[3], const int32_t *page_indptr, const int32_t *page_indices,
+                               const int32_t *suffix_lens, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return suffix_impl(plan, q, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens, workspace,
+                       workspace_bytes, cuda_stream, false);
+}
+
+static psa_status_t merge_impl(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream, bool after_stage)
 {
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
@@ -200,9 +211,16 @@ psa_status_t psa_decode_merge(const psa_plan_t *plan, const int32_t *suffix_lens
     a.num_q_heads = plan->cfg.num_q_heads; a.num_kv_heads = plan->cfg.num_kv_heads; a.head_dim = plan->cfg.head_dim;
     a.chunk_tokens = plan->suffix_chunk_tokens; a.out_dtype = plan->cfg.out_dtype;
     a.out = out; a.lse = lse;
+    a.after_stage = after_stage;
     std::string err;
     if (psa::launch_merge(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
     return PSA_OK;
+}
+
+psa_status_t psa_decode_merge(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse, void *workspace,
+                              size_t workspace_bytes, void *cuda_stream)
+{
+    return merge_impl(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream, false);
 }
 
 psa_status_t psa_decode(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,
@@ -213,10 +231,13 @@ psa_status_t psa_decode(const psa_plan_t *plan, const void *q, const void *prefi
 {
     psa_status_t st = psa_decode_prefix(plan, q, prefix_k, prefix_v, prefix_strides, workspace, workspace_bytes, cuda_stream);
     if (st != PSA_OK) return st;
-    st = psa_decode_suffix(plan, q, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens,
-                           workspace, workspace_bytes, cuda_stream);
+    // The suffix stage is independent of the prefix stage: launched as its programmatic dependent it runs
+    // beside it.  The merge stage needs both; the suffix blocks retire only after the prefix grid completed.
+    const bool have_prefix = !plan->prefix_items.empty(), have_suffix = !plan->suffix_items.empty();
+    st = suffix_impl(plan, q, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens, workspace,
+                     workspace_bytes, cuda_stream, have_prefix);
     if (st != PSA_OK) return st;
-    return psa_decode_merge(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream);
+    return merge_impl(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream, have_prefix || have_suffix);
 }
 
 namespace {

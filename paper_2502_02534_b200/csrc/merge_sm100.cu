@@ -48,6 +48,9 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
         return i < pre_splits ? pre_first + i * pre_split_stride : suf_first + (i - pre_splits) * group;
     };
 
+    // launched as a programmatic dependent: the partial results exist only after the preceding grids completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // pass 1: the largest lse (lanes stride over the partials)
     float top = -INFINITY;
     for (int i = lane; i < n_total; i += 32) top = fmaxf(top, __ldcg(partial_lse + partial_row(i)));
@@ -128,13 +131,23 @@ int launch_merge(const MergeArgs &a, void *stream, std::string *err)
     const int group = a.num_q_heads / a.num_kv_heads;
     const dim3 grid((rows + kMergeWarps - 1) / kMergeWarps), block(kMergeWarps * 32);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = a.after_stage ? 1 : 0;   // start filling in while the preceding stage drains
+    const int f32 = a.out_dtype == PSA_OUT_F32;
+    cudaError_t e;
     if (a.head_dim == 128)
-        merge_kernel<128><<<grid, block, 0, st>>>(a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
-                                                  a.num_q_heads, group, a.chunk_tokens, a.out_dtype == PSA_OUT_F32, a.out, a.lse);
+        e = cudaLaunchKernelEx(&lc, merge_kernel<128>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
     else
-        merge_kernel<64><<<grid, block, 0, st>>>(a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
-                                                 a.num_q_heads, group, a.chunk_tokens, a.out_dtype == PSA_OUT_F32, a.out, a.lse);
-    cudaError_t e = cudaGetLastError();
+        e = cudaLaunchKernelEx(&lc, merge_kernel<64>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
     if (e != cudaSuccess && err) *err = std::string("merge launch: ") + cudaGetErrorString(e);
     return int(e);
 }

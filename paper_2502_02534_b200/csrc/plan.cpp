@@ -86,6 +86,9 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     if (cfg.out_dtype != PSA_OUT_BF16 && cfg.out_dtype != PSA_OUT_F32)
         return fail(PSA_ERR_UNSUPPORTED, "out_dtype must be PSA_OUT_BF16 or PSA_OUT_F32");
     if (cfg.reserved != 0) return fail(PSA_ERR_INVALID_ARG, "reserved must be 0");
+    if (cfg.suffix_chunk_tokens < 0 || cfg.suffix_chunk_tokens % 64 != 0)
+        return fail(PSA_ERR_INVALID_ARG, "suffix_chunk_tokens must be 0 or a multiple of 64");
+    if (cfg.prefix_tiles_per_item < 0) return fail(PSA_ERR_INVALID_ARG, "prefix_tiles_per_item must be >= 0");
     if (cfg.num_sms <= 0) return fail(PSA_ERR_INVALID_ARG, "num_sms must be positive here");
     if (P < 0 || (P > 0 && (!prefix_lens || !n_samples))) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
 
@@ -115,7 +118,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
         tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;
         groups[p] = int64_t(cfg.num_kv_heads) * ceil_div(n_samples[p], samples_per_group);
     }
-    const int T = choose_prefix_tiles_per_item(tiles, groups, cfg.num_sms);
+    const int T = cfg.prefix_tiles_per_item > 0 ? cfg.prefix_tiles_per_item : choose_prefix_tiles_per_item(tiles, groups, cfg.num_sms);
     plan->prefix_tiles_per_item = T;
 
     plan->sample_info.assign(size_t(B), SampleInfo{});
@@ -166,6 +169,8 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
         samp_off += N;
     }
     plan->prefix_tiles_per_item = std::max(1, longest_item_tiles);
+    plan->prefix_max_rows_per_item = 0;
+    for (const PrefixItem &it : plan->prefix_items) plan->prefix_max_rows_per_item = std::max(plan->prefix_max_rows_per_item, it.n_rows);
     // longest items first: the hardware scheduler then fills the tail with short ones
     std::stable_sort(plan->prefix_items.begin(), plan->prefix_items.end(), [](const PrefixItem &a, const PrefixItem &b) {
         const int64_t ca = int64_t(ceil_div(a.n_keys, kPrefixTileKeys)) * (a.n_rows > kPrefixTileRows ? 2 : 1);
@@ -174,7 +179,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     });
 
     // ---- suffix items
-    const int C = choose_suffix_chunk(suffix_lens, int(B), cfg.num_kv_heads, cfg.num_sms);
+    const int C = cfg.suffix_chunk_tokens > 0 ? cfg.suffix_chunk_tokens : choose_suffix_chunk(suffix_lens, int(B), cfg.num_kv_heads, cfg.num_sms);
     plan->suffix_chunk_tokens = C;
     plan->suffix_items.clear();
     for (int64_t s = 0; s < B; ++s) {

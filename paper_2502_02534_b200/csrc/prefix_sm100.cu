@@ -10,15 +10,19 @@
 // (the result is unchanged: the factor cancels between O and l), so the accumulator in
 // TMEM is almost never rescaled.
 //
-// One thread block = one work item = (kv head, up to 256 query rows, a range of keys):
-//   warps 0-3   softmax warpgroup of row tile 0 (rows 0..127; thread = TMEM lane = row)
-//   warps 4-7   softmax warpgroup of row tile 1 (rows 128..255; idle when the item has <= 128 rows)
-//   warp  8     TMA producer: Q once, then K and V tiles of 128 keys through a ring of buffers
-//   warp  9     MMA issuer (one elected lane) and owner of the TMEM allocation
+// One thread block = one work item = (kv head, up to 256 query rows, a range of keys).
+// Two shapes of block, chosen per launch from the plan:
+//   two row tiles (some item has > 128 rows), 10 warps:
+//     warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1 (thread = TMEM lane = query row)
+//     warp 8           TMA producer: Q once, then K and V tiles of 128 keys through a ring of buffers
+//     warp 9           MMA issuer (one lane) and owner of the TMEM allocation
+//     The two row tiles alternate on the tensor pipe, so one tile's softmax overlaps the other's MMAs.
+//   one row tile (every item has <= 128 rows), 6 warps: warps 0-3 softmax, 4 producer, 5 MMA.
+//     The two S buffers alternate by key tile instead, so QK^T of tile j+1 runs under the softmax
+//     of tile j; the block is small enough to share an SM with a block of the suffix stage.
 // Per key tile and row tile:  S = Q K^T (SS MMA, K-major operands, 128-byte swizzle)
 // -> softmax warpgroup reads S from TMEM, writes P (bf16) over it -> O += P V (TS MMA,
-// P from TMEM, V as MN-major B operand).  The two row tiles alternate on the tensor pipe,
-// so one tile's softmax overlaps the other's MMAs; K/V are read from HBM/L2 once per item.
+// P from TMEM, V as MN-major B operand).  K/V are read from HBM/L2 once per item.
 //
 // Every wait on an mbarrier is bounded: when the limit passes, the block raises
 // PSA_ERR_TIMEOUT in the status word, stops storing results, and drains to a normal exit
@@ -34,11 +38,6 @@
 namespace psa {
 namespace {
 
-constexpr int kSoftmaxWarps = 8;
-constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
-constexpr int kThreads = 10 * 32;
-constexpr int kRing = 5;                 // K/V tile buffers in flight
 constexpr float kRescaleThreshold = 8.f; // log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
@@ -186,44 +185,55 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
            (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
 }
 
-template <int D>
+// Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 10 warps); otherwise one row
+// tile (one Q tile, 6 warps).  The ring length is chosen at launch.
+constexpr int kMaxRing = 6;
+template <int D, bool kTwo>
 struct PrefixSmem {
     static constexpr int kHalfBytes = kPrefixTileKeys * 128;          // one TMA box: 128 rows x 64 bf16
     static constexpr int kHalves = D / 64;
     static constexpr int kTileBytes = kHalves * kHalfBytes;           // a Q, K or V tile
-    static constexpr int kQOff = 0;                                   // 2 Q tiles
-    static constexpr int kRingOff = 2 * kTileBytes;
-    static constexpr int kBarOff = kRingOff + kRing * kTileBytes;
-    static constexpr int kNumBars = 1 + 2 * kRing + 6;               // q, full[], empty[], s_full[2], p_full[2], o_done[2]
+    static constexpr int kQTiles = kTwo ? 2 : 1;
+    static constexpr int kBarOff = 0;                                 // barriers first, tiles after them
+    static constexpr int kNumBars = 1 + 2 * kMaxRing + 4;             // q, full[], empty[], s_full[2], p_full[2]
     static constexpr int kTmemPtrOff = kBarOff + 8 * kNumBars;
     static constexpr int kAbortOff = kTmemPtrOff + 4;
-    static constexpr int kTotal = kAbortOff + 4 + 1024;               // + slack to align the base to 1024
+    static constexpr int kQOff = 1024;
+    static constexpr int kRingOff = kQOff + kQTiles * kTileBytes;
+    static constexpr int kStageRowFloats = D + 4;                     // padded row of the epilogue staging tile
+    static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;
     static constexpr int kTmemCols = 512;                             // S0 S1 (128 each) at 0, O0 O1 (D each) at 256
+    static constexpr int total(int ring) { return kRingOff + ring * kTileBytes; }
+    static constexpr int min_ring() { return (kQTiles * kStageBytes + kTileBytes - 1) / kTileBytes; }
 };
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, bool kTwo>
+__global__ void __launch_bounds__(kTwo ? 320 : 192, 1)
 prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
+              const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
               float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    using L = PrefixSmem<D>;
+    using L = PrefixSmem<D, kTwo>;
+    constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
+    constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
     constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
     constexpr int kPSteps = kPrefixTileKeys / 16;   // MMA k-steps of PV
     constexpr uint32_t kIdescQK = make_idesc(kPrefixTileKeys, false);
     constexpr uint32_t kIdescPV = make_idesc(D, true);
-    constexpr uint32_t kColS = 0, kColO = 2 * kPrefixTileKeys;   // S_t at t*128, O_t at 256 + t*D
+    constexpr uint32_t kColS = 0, kColO = 2 * kPrefixTileKeys;
 
-    extern __shared__ unsigned char smem_unaligned[];
-    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_unaligned) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {   // swizzled tiles need a 1024-byte aligned base; refuse to run rather than read garbage
+        if (threadIdx.x == 0) atomicCAS(status, 0, int(PSA_ERR_BOUNDS));
+        return;
+    }
     const uint32_t bar0 = sbase + L::kBarOff;
     auto bar_q = [&]() { return bar0; };
     auto bar_full = [&](int i) { return bar0 + 8 * (1 + i); };
-    auto bar_empty = [&](int i) { return bar0 + 8 * (1 + kRing + i); };
-    auto bar_s = [&](int t) { return bar0 + 8 * (1 + 2 * kRing + t); };
-    auto bar_p = [&](int t) { return bar0 + 8 * (3 + 2 * kRing + t); };
-    auto bar_o = [&](int t) { return bar0 + 8 * (5 + 2 * kRing + t); };
+    auto bar_empty = [&](int i) { return bar0 + 8 * (1 + kMaxRing + i); };
+    auto bar_s = [&](int b) { return bar0 + 8 * (1 + 2 * kMaxRing + b); };
+    auto bar_p = [&](int b) { return bar0 + 8 * (3 + 2 * kMaxRing + b); };
     volatile uint32_t *tmem_ptr = reinterpret_cast<volatile uint32_t *>(smem + L::kTmemPtrOff);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kAbortOff);
 
@@ -233,14 +243,19 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const int first_token = it0.x, n_keys = it0.y, kv = it0.z, first_sample = it0.w;
     const int n_rows = it1.x, prow0 = it1.y;
     const int n_tiles = (n_keys + kPrefixTileKeys - 1) / kPrefixTileKeys;
-    const int n_slots = n_rows > kPrefixTileRows ? 2 : 1;
+    const int n_rt = kTwo ? (n_rows > kPrefixTileRows ? 2 : 1) : 1;   // row tiles in use
     const int samples_per_tile = kPrefixTileRows / group;
+
+    // Which S buffer / barrier phase serves (row tile t, key tile j):
+    //   two row tiles: buffer t, one use per key tile;  one row tile: buffers alternate with j.
+    auto sbuf = [&](int t, int j) { return kTwo ? t : (j & 1); };
+    auto sphase = [&](int j) { return uint32_t(kTwo ? (j & 1) : ((j >> 1) & 1)); };
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         mbar_init(bar_q(), 1);
-        for (int i = 0; i < kRing; ++i) { mbar_init(bar_full(i), 1); mbar_init(bar_empty(i), 1); }
-        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128); mbar_init(bar_o(t), 1); }
+        for (int i = 0; i < kMaxRing; ++i) { mbar_init(bar_full(i), 1); mbar_init(bar_empty(i), 1); }
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128); }
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
@@ -252,18 +267,20 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
+    // every block is resident now: a kernel launched as a programmatic dependent may start filling the machine
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            mbar_expect_tx(bar_q(), n_slots * L::kTileBytes);
-            for (int t = 0; t < n_slots; ++t)
+            mbar_expect_tx(bar_q(), n_rt * L::kTileBytes);
+            for (int t = 0; t < n_rt; ++t)
                 for (int h = 0; h < L::kHalves; ++h)
                     tma_load_4d(sbase + L::kQOff + t * L::kTileBytes + h * L::kHalfBytes, &map_q, bar_q(), h * 64, 0, kv,
                                 first_sample + t * samples_per_tile);
             // ring order: K0 V0 K1 V1 ...
             for (int i = 0; i < 2 * n_tiles; ++i) {
-                const int slot = i % kRing, use = i / kRing;
+                const int slot = i % ring, use = i / ring;
                 if (use > 0 && !mbar_wait(bar_empty(slot), (use - 1) & 1, abort_flag)) break;
                 const int tok = first_token + (i >> 1) * kPrefixTileKeys;
                 const CUtensorMap *map = (i & 1) ? &map_v : &map_k;
@@ -276,59 +293,85 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool ok = mbar_wait(bar_q(), 0, abort_flag);
-            auto issue_qk = [&](int t, int j) {   // S_t = Q_t K_j^T ; K_j is ring entry 2j
-                const int slot = (2 * j) % kRing;
+            auto wait_entry = [&](int e) { return mbar_wait(bar_full(e % ring), (e / ring) & 1, abort_flag); };
+            auto issue_qk = [&](int t, int j) {   // S[sbuf] = Q_t K_j^T ; K_j is ring entry 2j
                 const uint32_t qa = sbase + L::kQOff + t * L::kTileBytes;
-                const uint32_t kb = sbase + L::kRingOff + slot * L::kTileBytes;
+                const uint32_t kb = sbase + L::kRingOff + ((2 * j) % ring) * L::kTileBytes;
+                const uint32_t d = tmem_base + kColS + sbuf(t, j) * kPrefixTileKeys;
 #pragma unroll
                 for (int k = 0; k < kKSteps; ++k) {
                     const uint32_t off = (k / 4) * L::kHalfBytes + (k % 4) * 32;
-                    mma_ss(tmem_base + kColS + t * kPrefixTileKeys, make_smem_desc(qa + off, 16, 1024),
-                           make_smem_desc(kb + off, 16, 1024), kIdescQK, k > 0);
+                    mma_ss(d, make_smem_desc(qa + off, 16, 1024), make_smem_desc(kb + off, 16, 1024), kIdescQK, k > 0);
                 }
             };
-            auto issue_pv = [&](int t, int j) {   // O_t += P_t V_j ; V_j is ring entry 2j+1
-                const int slot = (2 * j + 1) % kRing;
-                const uint32_t vb = sbase + L::kRingOff + slot * L::kTileBytes;
+            auto issue_pv = [&](int t, int j) {   // O_t += P[sbuf] V_j ; V_j is ring entry 2j+1
+                const uint32_t vb = sbase + L::kRingOff + ((2 * j + 1) % ring) * L::kTileBytes;
+                const uint32_t a = tmem_base + kColS + sbuf(t, j) * kPrefixTileKeys;
 #pragma unroll
                 for (int k = 0; k < kPSteps; ++k)
-                    mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kPrefixTileKeys + k * 8,
-                           make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV, (j > 0 || k > 0));
+                    mma_ts(tmem_base + kColO + t * D, a + k * 8, make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV,
+                           (j > 0 || k > 0));
             };
-            if (ok) ok = mbar_wait(bar_full(0), 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                for (int t = 0; t < n_slots; ++t) { issue_qk(t, 0); tc_commit(bar_s(t)); }
-            }
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const int vslot = (2 * j + 1) % kRing, kslot = (2 * j) % kRing;
-                if (!(ok = mbar_wait(bar_full(vslot), ((2 * j + 1) / kRing) & 1, abort_flag))) break;
-                if (j + 1 < n_tiles) {
-                    const int nslot = (2 * j + 2) % kRing;
-                    if (!(ok = mbar_wait(bar_full(nslot), ((2 * j + 2) / kRing) & 1, abort_flag))) break;
-                }
-                for (int t = 0; t < n_slots; ++t) {
-                    if (!(ok = mbar_wait(bar_p(t), j & 1, abort_flag))) break;
+            if constexpr (kTwo) {
+                if (ok) ok = wait_entry(0);
+                if (ok) {
                     tc_fence_after();
-                    issue_pv(t, j);
-                    if (t == n_slots - 1) { tc_commit(bar_empty(kslot)); tc_commit(bar_empty(vslot)); }
-                    if (j + 1 < n_tiles) { issue_qk(t, j + 1); tc_commit(bar_s(t)); }
-                    else tc_commit(bar_o(t));
+                    for (int t = 0; t < n_rt; ++t) { issue_qk(t, 0); tc_commit(bar_s(t)); }
+                    tc_commit(bar_empty(0));                       // K_0 is free once both QK^T are done
+                }
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    if (!(ok = wait_entry(2 * j + 1))) break;
+                    if (j + 1 < n_tiles && !(ok = wait_entry(2 * j + 2))) break;
+                    for (int t = 0; t < n_rt; ++t) {
+                        if (!(ok = mbar_wait(bar_p(t), sphase(j), abort_flag))) break;
+                        tc_fence_after();
+                        issue_pv(t, j);
+                        if (t == n_rt - 1) tc_commit(bar_empty((2 * j + 1) % ring));
+                        if (j + 1 < n_tiles) {
+                            issue_qk(t, j + 1);
+                            tc_commit(bar_s(t));
+                            if (t == n_rt - 1) tc_commit(bar_empty((2 * j + 2) % ring));
+                        }
+                    }
+                }
+            } else {
+                // one row tile: S0/S1 alternate by key tile, so QK^T of tile j+1 runs under the softmax of tile j
+                for (int j = 0; ok && j < 2 && j < n_tiles; ++j) {
+                    if (!(ok = wait_entry(2 * j))) break;
+                    tc_fence_after();
+                    issue_qk(0, j);
+                    tc_commit(bar_s(j & 1));
+                    tc_commit(bar_empty((2 * j) % ring));
+                }
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    if (!(ok = wait_entry(2 * j + 1))) break;
+                    if (!(ok = mbar_wait(bar_p(j & 1), sphase(j), abort_flag))) break;
+                    tc_fence_after();
+                    issue_pv(0, j);
+                    tc_commit(bar_empty((2 * j + 1) % ring));
+                    if (j + 2 < n_tiles) {
+                        if (!(ok = wait_entry(2 * j + 4))) break;
+                        tc_fence_after();
+                        issue_qk(0, j + 2);
+                        tc_commit(bar_s(j & 1));
+                        tc_commit(bar_empty((2 * j + 4) % ring));
+                    }
                 }
             }
         }
-    } else if (warp < 4 * n_slots) {
+    } else if (warp < 4 * n_rt) {
         // ------------------------------------------------------------ softmax + epilogue
         const int t = warp >> 2;                       // row tile
         const int row = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
         const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t s_addr = tmem_base + lane_addr + kColS + t * kPrefixTileKeys;
         const uint32_t o_addr = tmem_base + lane_addr + kColO + t * D;
         float m_ref = -INFINITY, l_sum = 0.f;
         bool ok = true;
         uint32_t sreg[4][32];
         for (int j = 0; j < n_tiles; ++j) {
-            if (!(ok = mbar_wait(bar_s(t), j & 1, abort_flag))) break;
+            const int b = sbuf(t, j);
+            const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kPrefixTileKeys;
+            if (!(ok = mbar_wait(bar_s(b), sphase(j), abort_flag))) break;
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
@@ -357,7 +400,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const float m_new = need ? tmax : m_ref;
                 const float alpha = need ? fast_exp2(m_ref - m_new) : 1.f;   // 0 on the first tile
                 if (j > 0) {
-                    // s_full of tile j was committed after PV of tile j-1: O is quiescent until P of tile j is handed over
+                    // O must be quiescent: PV of tile j-1 has to be complete, which is what releases the ring
+                    // buffer of V_{j-1} (PV of tile j cannot start before this thread hands over P)
+                    if (!(ok = mbar_wait(bar_empty((2 * j - 1) % ring), ((2 * j - 1) / ring) & 1, abort_flag))) break;
+                    tc_fence_after();
                     uint32_t oreg[32];
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
@@ -389,29 +435,43 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             tmem_st32(s_addr + 32, sreg[1]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_p(t));
+            mbar_arrive(bar_p(b));
         }
-        // ---- epilogue: out = O / l, lse = (m + log2 l) ln 2
-        if (ok) ok = mbar_wait(bar_o(t), 0, abort_flag);
+        // ---- epilogue: out = O / l, lse = (m + log2 l) ln 2.  The tile goes through shared memory (the
+        // ring is idle by now) so that every global store instruction writes one full 4*D-byte row.
+        // The release of the last V buffer follows the last MMA of the block (of both row tiles): O is final
+        // and nothing reads the ring any more, so the staging tile may overlay it.
+        if (ok) ok = mbar_wait(bar_empty((2 * n_tiles - 1) % ring), ((2 * n_tiles - 1) / ring) & 1, abort_flag);
+        float *stage = reinterpret_cast<float *>(smem + L::kRingOff + t * L::kStageBytes);
         if (ok) {
             tc_fence_after();
-            const int r = t * kPrefixTileRows + row;
             const float inv = 1.f / l_sum;
-            float *dst = partial_o + size_t(prow0 + r) * D;
+            float *mine = stage + row * L::kStageRowFloats;
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t oreg[32];
                 tmem_ld32(o_addr + c * 32, oreg);
                 tmem_wait_ld();
-                if (r < n_rows) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<float4 *>(dst + c * 32 + i) =
-                            make_float4(__uint_as_float(oreg[i]) * inv, __uint_as_float(oreg[i + 1]) * inv,
-                                        __uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
-                }
+                for (int i = 0; i < 32; i += 4)
+                    *reinterpret_cast<float4 *>(mine + c * 32 + i) =
+                        make_float4(__uint_as_float(oreg[i]) * inv, __uint_as_float(oreg[i + 1]) * inv,
+                                    __uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
             }
+            const int r = t * kPrefixTileRows + row;
             if (r < n_rows) partial_lse[prow0 + r] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+        }
+        // the four warps of this row tile meet (named barrier 1 + t), then write rows round-robin
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+        if (!*abort_flag) {
+            constexpr int kLanesPerRow = D / 4;                    // float4 per row: 32 or 16
+            constexpr int kRowsPerInstr = 32 / kLanesPerRow;       // 1 or 2
+            const int sub = lane / kLanesPerRow, col = (lane % kLanesPerRow) * 4;
+            const int rows_here = min(kPrefixTileRows, n_rows - t * kPrefixTileRows);
+            for (int r = (warp & 3) * kRowsPerInstr + sub; r < rows_here; r += 4 * kRowsPerInstr) {
+                const float4 v = *reinterpret_cast<const float4 *>(stage + r * L::kStageRowFloats + col);
+                *reinterpret_cast<float4 *>(partial_o + size_t(prow0 + t * kPrefixTileRows + r) * D + col) = v;
+            }
         }
     }
 
@@ -467,20 +527,29 @@ bool encode(EncodeFn fn, CUtensorMap *map, const void *base, int rank, const cuu
     return true;
 }
 
-template <int D>
+template <int D, bool kTwo>
 int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
 {
-    using L = PrefixSmem<D>;
-    auto kern = prefix_kernel<D>;
+    using L = PrefixSmem<D, kTwo>;
+    auto kern = prefix_kernel<D, kTwo>;
+    // ring length: enough buffers for the epilogue staging tile(s); short items of the one-row-tile
+    // shape get the smallest block so that a suffix block fits beside it on the SM
+    constexpr int kLongRing = (kTwo && D == 128) ? 5 : kMaxRing;   // the longest ring that fits in 227 KB
+    static_assert(L::total(kLongRing) <= 227 * 1024 && L::min_ring() <= kLongRing, "shared memory plan does not fit");
+    int ring = (!kTwo && D == 128 && a.max_tiles_per_item <= 2) ? 3 : kLongRing;
+    ring = ring < L::min_ring() ? L::min_ring() : ring;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total(kLongRing));
+        if (e != cudaSuccess) return int(e);
+        // ask for the largest shared-memory carve-out so that a suffix block can share the SM
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return int(e);
         configured = true;
     }
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
-    kern<<<a.num_items, kThreads, L::kTotal, st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, scale_log2,
-                                                   a.partial_o, a.partial_lse, a.status);
+    kern<<<a.num_items, kTwo ? 320 : 192, L::total(ring), st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, ring,
+                                                               scale_log2, a.partial_o, a.partial_lse, a.status);
     return int(cudaGetLastError());
 }
 
@@ -508,7 +577,9 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
         if (!encode(fn, &mv, a.v, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int rc = D == 128 ? launch_one<128>(a, mq, mk, mv, st) : launch_one<64>(a, mq, mk, mv, st);
+    int rc;
+    if (a.max_rows_per_item > kPrefixTileRows) rc = D == 128 ? launch_one<128, true>(a, mq, mk, mv, st) : launch_one<64, true>(a, mq, mk, mv, st);
+    else rc = D == 128 ? launch_one<128, false>(a, mq, mk, mv, st) : launch_one<64, false>(a, mq, mk, mv, st);
     if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));
     return rc;
 }

@@ -78,6 +78,7 @@ struct psa_plan {
     std::vector<psa::SuffixItem> suffix_items;
     std::vector<psa::SampleInfo> sample_info;
     int32_t prefix_tiles_per_item = 0;
+    int32_t prefix_max_rows_per_item = 0;
     int32_t suffix_chunk_tokens = 0;
     int64_t num_partial_rows = 0;
     psa::WorkspaceLayout ws;
@@ -102,6 +103,7 @@ struct PrefixArgs {
     float sm_scale;
     const PrefixItem *items;  // device
     int32_t num_items;
+    int32_t max_rows_per_item, max_tiles_per_item;  // over all items of the plan
     float *partial_o, *partial_lse;  // device
     int32_t *status;                 // device
 };
@@ -118,6 +120,7 @@ struct SuffixArgs {
     int32_t num_items, chunk_tokens;
     float *partial_o, *partial_lse;
     int32_t *status;
+    bool after_prefix = false;  // launched right behind the prefix stage of the same step: may overlap it
 };
 int launch_suffix(const SuffixArgs &a, void *stream, std::string *err);
 
@@ -128,6 +131,7 @@ struct MergeArgs {
     int32_t num_samples, num_q_heads, num_kv_heads, head_dim, chunk_tokens, out_dtype;
     void *out;
     float *lse;
+    bool after_stage = false;  // launched right behind a prefix / suffix stage of the same step
 };
 int launch_merge(const MergeArgs &a, void *stream, std::string *err);
 

@@ -101,7 +101,10 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     int S = __ldg(suffix_lens + s);
     S = min(S, __ldg(&sample_info[s].suf_len_bound));
     const int n_tok = min(S - tok0, chunk_tokens);
-    if (n_tok <= 0) return;  // the merge stage derives the chunk count from the same length
+    if (n_tok <= 0) {  // the merge stage derives the chunk count from the same length
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     const int n_pages = (n_tok + kPageSize - 1) / kPageSize;
     const int my_pages = (n_pages - warp + kWarps - 1) / kWarps;  // pages warp, warp+4, ...
     const int32_t *my_page_ids = page_indices + __ldg(page_indptr + s) + tok0 / kPageSize;
@@ -254,6 +257,11 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
         partial_o[size_t(prow0 + g) * D + d] = acc / z;
         if (d == 0) partial_lse[prow0 + g] = (top + log2f(z)) * 0.6931471805599453f;
     }
+    // When launched as a programmatic dependent of the prefix stage this grid runs beside it.  The merge
+    // stage may be scheduled once every block is here, and no block retires before the prefix grid has
+    // completed, so that "suffix grid complete" implies "prefix grid complete" for the merge stage.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 template <int D, int G>
@@ -266,15 +274,25 @@ int launch_one(const SuffixArgs &a, cudaStream_t st)
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
         if (e != cudaSuccess) return int(e);
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return int(e);
         configured = true;
     }
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
-    kern<<<a.num_items, kWarps * 32, L::kTotal, st>>>(
-        static_cast<const __nv_bfloat16 *>(a.q), static_cast<const __nv_bfloat16 *>(a.pool_k),
-        static_cast<const __nv_bfloat16 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok, a.page_indptr,
-        a.page_indices, a.suffix_lens, a.items, a.sample_info, a.num_q_heads, a.chunk_tokens, scale_log2, a.partial_o,
-        a.partial_lse);
-    return int(cudaGetLastError());
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(a.num_items);
+    lc.blockDim = dim3(kWarps * 32);
+    lc.dynamicSmemBytes = L::kTotal;
+    lc.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = a.after_prefix ? 1 : 0;   // run beside the prefix stage launched just before
+    return int(cudaLaunchKernelEx(&lc, kern, static_cast<const __nv_bfloat16 *>(a.q), static_cast<const __nv_bfloat16 *>(a.pool_k),
+                                  static_cast<const __nv_bfloat16 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok,
+                                  a.page_indptr, a.page_indices, a.suffix_lens, a.items, a.sample_info, a.num_q_heads,
+                                  a.chunk_tokens, scale_log2, a.partial_o, a.partial_lse));
 }
 
 }  // namespace
