@@ -58,7 +58,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
     for (int o = 16; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, o));
 
     // pass 2: lane i of each group of 32 partials computes weight and row; the rows are then
-    // fetched four at a time so that several loads are in flight per lane
+    // fetched eight at a time so that several loads are in flight per lane
     float acc[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = 0.f;
@@ -81,15 +81,25 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
             z += my_w;
             const int cnt = min(32, n_total - base);
             int i = 0;
-            for (; i + 4 <= cnt; i += 4) {
-                float4 x[4]; float w[4];
+            for (; i + 8 <= cnt; i += 8) {
+                float4 x[8]; float w[8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     w[u] = __shfl_sync(0xffffffffu, my_w, i + u);
                     x[u] = fetch(__shfl_sync(0xffffffffu, my_row, i + u));
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) fma_row(w[u], x[u]);
+                for (int u = 0; u < 8; ++u) fma_row(w[u], x[u]);
+            }
+            for (; i + 2 <= cnt; i += 2) {
+                float4 x[2]; float w[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    w[u] = __shfl_sync(0xffffffffu, my_w, i + u);
+                    x[u] = fetch(__shfl_sync(0xffffffffu, my_row, i + u));
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) fma_row(w[u], x[u]);
             }
             for (; i < cnt; ++i) {
                 const float w = __shfl_sync(0xffffffffu, my_w, i);

@@ -46,10 +46,13 @@ int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::v
 }
 
 // Suffix: items are dispatched greedily to 2 resident blocks per SM.  Estimate =
-// (sum of item costs) / slots + cost of one full item (the tail); cost = tokens + 64.
+// (sum of item costs) / slots + cost of one full item (the tail); cost = tokens + 384: a block
+// spends about as long finding its pages (three dependent loads) and combining its warps as it
+// spends streaming 384 tokens (measured on B200: 512-token chunks beat 128-token chunks by 30 %
+// on 32 samples x U[0,1024] tokens).
 int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sms)
 {
-    const double overhead = 64.0;
+    const double overhead = 384.0;
     const double slots = 2.0 * num_sms;
     double best_cost = std::numeric_limits<double>::infinity();
     int best = 64;

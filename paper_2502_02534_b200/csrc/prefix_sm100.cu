@@ -149,6 +149,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
                    "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
                  : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -207,11 +214,11 @@ struct PrefixSmem {
     static constexpr int min_ring() { return (kQTiles * kStageBytes + kTileBytes - 1) / kTileBytes; }
 };
 
-template <int D, bool kTwo>
-__global__ void __launch_bounds__(kTwo ? 320 : 192, 1)
-prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
-              float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+template <int D, bool kTwo, bool kLowReg>
+__device__ __forceinline__ void
+prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensorMap *pmap_v,
+            const PrefixItem *__restrict__ items, int group, int ring, float scale_log2,
+            float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
     using L = PrefixSmem<D, kTwo>;
     constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
@@ -262,7 +269,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_ptr)), L::kTmemCols);
         tmem_relinquish();
     }
-    if (warp == kProducerWarp && lane == 0) { prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }
+    if (warp == kProducerWarp && lane == 0) { prefetch_tensormap(pmap_q); prefetch_tensormap(pmap_k); prefetch_tensormap(pmap_v); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -276,14 +283,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             mbar_expect_tx(bar_q(), n_rt * L::kTileBytes);
             for (int t = 0; t < n_rt; ++t)
                 for (int h = 0; h < L::kHalves; ++h)
-                    tma_load_4d(sbase + L::kQOff + t * L::kTileBytes + h * L::kHalfBytes, &map_q, bar_q(), h * 64, 0, kv,
+                    tma_load_4d(sbase + L::kQOff + t * L::kTileBytes + h * L::kHalfBytes, pmap_q, bar_q(), h * 64, 0, kv,
                                 first_sample + t * samples_per_tile);
             // ring order: K0 V0 K1 V1 ...
             for (int i = 0; i < 2 * n_tiles; ++i) {
                 const int slot = i % ring, use = i / ring;
                 if (use > 0 && !mbar_wait(bar_empty(slot), (use - 1) & 1, abort_flag)) break;
                 const int tok = first_token + (i >> 1) * kPrefixTileKeys;
-                const CUtensorMap *map = (i & 1) ? &map_v : &map_k;
+                const CUtensorMap *map = (i & 1) ? pmap_v : pmap_k;
                 mbar_expect_tx(bar_full(slot), L::kTileBytes);
                 for (int h = 0; h < L::kHalves; ++h)
                     tma_load_3d(sbase + L::kRingOff + slot * L::kTileBytes + h * L::kHalfBytes, map, bar_full(slot), h * 64, kv, tok);
@@ -373,24 +380,32 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kPrefixTileKeys;
             if (!(ok = mbar_wait(bar_s(b), sphase(j), abort_flag))) break;
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
-            tmem_wait_ld();
             const int valid = n_keys - j * kPrefixTileKeys;   // >= 1; < 128 only on the last tile
             float tmax = -INFINITY;
-            if (valid >= kPrefixTileKeys) {
+            if constexpr (!kLowReg) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sreg[c][i]));
-            } else {
+                for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
+                tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;   // -inf: masked key
+                        if (valid < kPrefixTileKeys && c * 32 + i >= valid) sreg[c][i] = 0xff800000u;   // -inf: masked key
                         tmax = fmaxf(tmax, __uint_as_float(sreg[c][i]));
                     }
+            } else {
+                // low-register form: S is read twice from TMEM, 32 columns at a time (pass 1: maximum)
+                uint32_t r[2][32];
+                tmem_ld32(s_addr, r[0]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (valid >= kPrefixTileKeys || c * 32 + i < valid) tmax = fmaxf(tmax, __uint_as_float(r[c & 1][i]));
+                    tmem_wait_ld();
+                }
             }
             tmax *= scale_log2;
             // Move the reference maximum only when needed; the whole warp takes the slow path together
@@ -420,19 +435,44 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             }
             // p = 2^(c*s - m_ref); row sum from the fp32 values; P packed to bf16 over the first 64 columns of S
             float psum = 0.f;
+            if constexpr (!kLowReg) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 4; ++c) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_ref));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_ref));
-                    psum += p0 + p1;
-                    sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_ref));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_ref));
+                        psum += p0 + p1;
+                        sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                    }
+                }
+                tmem_st32(s_addr, sreg[0]);
+                tmem_st32(s_addr + 32, sreg[1]);
+            } else {
+                // pass 2: chunk c of S (columns 32c..32c+31) becomes columns 16c..16c+15 of P, which were read already
+                uint32_t r[2][32];
+                tmem_ld32(s_addr, r[0]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_ref));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_ref));
+                        if (valid < kPrefixTileKeys) {
+                            if (c * 32 + i >= valid) p0 = 0.f;
+                            if (c * 32 + i + 1 >= valid) p1 = 0.f;
+                        }
+                        psum += p0 + p1;
+                        pk[i / 2] = pack_bf16(p0, p1);
+                    }
+                    tmem_wait_ld();            // chunk c+1 has landed before P overwrites columns below it
+                    tmem_st16(s_addr + c * 16, pk);
                 }
             }
             l_sum += psum;
-            tmem_st32(s_addr, sreg[0]);
-            tmem_st32(s_addr + 32, sreg[1]);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p(b));
@@ -493,6 +533,36 @@ prefix_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     }
 }
 
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+{
+    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+}
+
+// 152 registers per thread: two of these warps and one suffix warp (208) fill the 512 registers per lane of
+// an SM sub-partition, which is what lets a suffix block run beside this block.
+template <int D>
+__global__ void __maxnreg__(152)
+prefix_kernel_one(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+{
+    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+}
+
+// One row tile, long items: the block owns the SM anyway (long ring), so S stays in registers.
+template <int D>
+__global__ void __launch_bounds__(192, 1)
+prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                       float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+{
+    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+}
+
 // ---------------------------------------------------------------- host side
 using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -527,16 +597,18 @@ bool encode(EncodeFn fn, CUtensorMap *map, const void *base, int rank, const cuu
     return true;
 }
 
-template <int D, bool kTwo>
+// kShape: 2 = two row tiles, 1 = one row tile with short items (small block), 0 = one row tile with long items
+template <int D, int kShape>
 int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
 {
+    constexpr bool kTwo = kShape == 2;
     using L = PrefixSmem<D, kTwo>;
-    auto kern = prefix_kernel<D, kTwo>;
+    auto kern = kShape == 2 ? prefix_kernel_two<D> : (kShape == 1 ? prefix_kernel_one<D> : prefix_kernel_one_long<D>);
     // ring length: enough buffers for the epilogue staging tile(s); short items of the one-row-tile
     // shape get the smallest block so that a suffix block fits beside it on the SM
     constexpr int kLongRing = (kTwo && D == 128) ? 5 : kMaxRing;   // the longest ring that fits in 227 KB
     static_assert(L::total(kLongRing) <= 227 * 1024 && L::min_ring() <= kLongRing, "shared memory plan does not fit");
-    int ring = (!kTwo && D == 128 && a.max_tiles_per_item <= 2) ? 3 : kLongRing;
+    int ring = kShape == 1 ? 3 : kLongRing;
     ring = ring < L::min_ring() ? L::min_ring() : ring;
     static bool configured = false;
     if (!configured) {
@@ -578,8 +650,9 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc;
-    if (a.max_rows_per_item > kPrefixTileRows) rc = D == 128 ? launch_one<128, true>(a, mq, mk, mv, st) : launch_one<64, true>(a, mq, mk, mv, st);
-    else rc = D == 128 ? launch_one<128, false>(a, mq, mk, mv, st) : launch_one<64, false>(a, mq, mk, mv, st);
+    if (a.max_rows_per_item > kPrefixTileRows) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
+    else if (a.max_tiles_per_item <= 2) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
+    else rc = D == 128 ? launch_one<128, 0>(a, mq, mk, mv, st) : launch_one<64, 0>(a, mq, mk, mv, st);
     if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));
     return rc;
 }
