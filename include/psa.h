@@ -70,6 +70,7 @@ typedef struct {
     int32_t num_sms;    /* SMs to plan for; 0 = ask the current CUDA device */
     int32_t suffix_chunk_tokens;   /* tokens per suffix work item: 0 = planner's choice, else a multiple of 64 */
     int32_t prefix_tiles_per_item; /* 128-key tiles per prefix work item: 0 = planner's choice */
+    int32_t prefix_rows_per_item;  /* query rows per prefix work item: 0 = planner's choice, else 128 or 256 */
     int32_t reserved;   /* must be 0 */
 } psa_config_t;
 

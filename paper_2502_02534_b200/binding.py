@@ -32,7 +32,7 @@ class PsaError(RuntimeError):
 class _Config(ctypes.Structure):
     _fields_ = [("num_q_heads", c_int32), ("num_kv_heads", c_int32), ("head_dim", c_int32), ("page_size", c_int32),
                 ("sm_scale", c_float), ("out_dtype", c_int32), ("num_sms", c_int32), ("suffix_chunk_tokens", c_int32),
-                ("prefix_tiles_per_item", c_int32), ("reserved", c_int32)]
+                ("prefix_tiles_per_item", c_int32), ("prefix_rows_per_item", c_int32), ("reserved", c_int32)]
 
 
 class _Info(ctypes.Structure):
@@ -139,14 +139,15 @@ class Plan:
     """psa_plan_create / psa_plan_destroy, plus the workspace the plan needs (a torch uint8 tensor)."""
 
     def __init__(self, prefix_lens, n_samples_per_prefix, suffix_lens, *, num_q_heads, num_kv_heads, head_dim,
-                 page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0, suffix_chunk_tokens=0, prefix_tiles_per_item=0):
+                 page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0, suffix_chunk_tokens=0, prefix_tiles_per_item=0,
+                 prefix_rows_per_item=0):
         lib = library()
         self.prefix_lens, self.n_samples, self.suffix_len_bounds = _i32(prefix_lens), _i32(n_samples_per_prefix), _i32(suffix_lens)
         self.num_q_heads, self.num_kv_heads, self.head_dim, self.page_size = num_q_heads, num_kv_heads, head_dim, page_size
         self.sm_scale = float(sm_scale if sm_scale is not None else head_dim ** -0.5)
         self.out_dtype = {"bf16": PSA_OUT_BF16, "f32": PSA_OUT_F32}[out_dtype]
         cfg = _Config(num_q_heads, num_kv_heads, head_dim, page_size, self.sm_scale, self.out_dtype, num_sms,
-                      suffix_chunk_tokens, prefix_tiles_per_item, 0)
+                      suffix_chunk_tokens, prefix_tiles_per_item, prefix_rows_per_item, 0)
         handle = c_void_p()
         self._h = None
         _check(lib.psa_plan_create(ctypes.byref(cfg), len(self.prefix_lens), _ptr(self.prefix_lens), _ptr(self.n_samples),

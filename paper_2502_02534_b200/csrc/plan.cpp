@@ -92,6 +92,8 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     if (cfg.suffix_chunk_tokens < 0 || cfg.suffix_chunk_tokens % 64 != 0)
         return fail(PSA_ERR_INVALID_ARG, "suffix_chunk_tokens must be 0 or a multiple of 64");
     if (cfg.prefix_tiles_per_item < 0) return fail(PSA_ERR_INVALID_ARG, "prefix_tiles_per_item must be >= 0");
+    if (cfg.prefix_rows_per_item != 0 && cfg.prefix_rows_per_item != 128 && cfg.prefix_rows_per_item != 256)
+        return fail(PSA_ERR_INVALID_ARG, "prefix_rows_per_item must be 0, 128 or 256");
     if (cfg.num_sms <= 0) return fail(PSA_ERR_INVALID_ARG, "num_sms must be positive here");
     if (P < 0 || (P > 0 && (!prefix_lens || !n_samples))) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
 
@@ -115,7 +117,14 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     plan->suffix_len_bounds.assign(suffix_lens, suffix_lens + B);
 
     // ---- prefix items
-    const int samples_per_group = kPrefixRowsPerItem / G;  // samples in one 256-row group
+    // Rows per item.  Two row tiles (256 rows) per block halve the K/V traffic into the SM, which pays once
+    // the stage is tensor-bound (R_p >= 512, above the machine's flop/byte ridge); below that a block of
+    // one row tile is small enough to share its SM with a suffix block, and the overlap is worth more.
+    int64_t max_rows = 0;
+    for (int p = 0; p < P; ++p) max_rows = std::max<int64_t>(max_rows, int64_t(n_samples[p]) * G);
+    const int rows_per_item = cfg.prefix_rows_per_item > 0 ? cfg.prefix_rows_per_item
+                                                           : (max_rows >= 2 * kPrefixRowsPerItem ? kPrefixRowsPerItem : kPrefixTileRows);
+    const int samples_per_group = rows_per_item / G;
     std::vector<int64_t> tiles(P), groups(P);
     for (int p = 0; p < P; ++p) {
         tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;

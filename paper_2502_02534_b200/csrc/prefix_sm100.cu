@@ -193,8 +193,12 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 }
 
 // Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 10 warps); otherwise one row
-// tile (one Q tile, 6 warps).  The ring length is chosen at launch.
+// tile (one Q tile, 6 warps).
 constexpr int kMaxRing = 6;
+// Ring length per block shape: 5 x 32 KB beside two Q tiles, 6 when the block owns the SM, 3 for the small
+// block that shares the SM with a suffix block (never fewer buffers than the epilogue staging tile needs).
+template <int D, bool kTwo, bool kLowReg>
+__host__ __device__ constexpr int prefix_ring() { return kLowReg ? 3 : ((kTwo && D == 128) ? 5 : kMaxRing); }
 template <int D, bool kTwo>
 struct PrefixSmem {
     static constexpr int kHalfBytes = kPrefixTileKeys * 128;          // one TMA box: 128 rows x 64 bf16
@@ -210,17 +214,18 @@ struct PrefixSmem {
     static constexpr int kStageRowFloats = D + 4;                     // padded row of the epilogue staging tile
     static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;
     static constexpr int kTmemCols = 512;                             // S0 S1 (128 each) at 0, O0 O1 (D each) at 256
-    static constexpr int total(int ring) { return kRingOff + ring * kTileBytes; }
-    static constexpr int min_ring() { return (kQTiles * kStageBytes + kTileBytes - 1) / kTileBytes; }
+    __host__ __device__ static constexpr int total(int ring) { return kRingOff + ring * kTileBytes; }
+    __host__ __device__ static constexpr int min_ring() { return (kQTiles * kStageBytes + kTileBytes - 1) / kTileBytes; }
 };
 
 template <int D, bool kTwo, bool kLowReg>
 __device__ __forceinline__ void
 prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensorMap *pmap_v,
-            const PrefixItem *__restrict__ items, int group, int ring, float scale_log2,
+            const PrefixItem *__restrict__ items, int group, float scale_log2,
             float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
     using L = PrefixSmem<D, kTwo>;
+    constexpr int ring = prefix_ring<D, kTwo, kLowReg>();   // K/V tile buffers in flight
     constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
     constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
     constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
@@ -386,26 +391,39 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
                 tmem_wait_ld();
+                float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (valid < kPrefixTileKeys) {   // last tile of a ragged prompt: masked keys become -inf
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;
+                }
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (valid < kPrefixTileKeys && c * 32 + i >= valid) sreg[c][i] = 0xff800000u;   // -inf: masked key
-                        tmax = fmaxf(tmax, __uint_as_float(sreg[c][i]));
-                    }
+                    for (int i = 0; i < 32; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(sreg[c][i]));   // eight independent chains
+                tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
             } else {
                 // low-register form: S is read twice from TMEM, 32 columns at a time (pass 1: maximum)
                 uint32_t r[2][32];
+                float mx[2] = {-INFINITY, -INFINITY};
                 tmem_ld32(s_addr, r[0]);
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+                    if (valid >= kPrefixTileKeys) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (valid >= kPrefixTileKeys || c * 32 + i < valid) tmax = fmaxf(tmax, __uint_as_float(r[c & 1][i]));
+                        for (int i = 0; i < 32; ++i) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (c * 32 + i < valid) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
+                    }
                     tmem_wait_ld();
                 }
+                tmax = fmaxf(mx[0], mx[1]);
             }
             tmax *= scale_log2;
             // Move the reference maximum only when needed; the whole warp takes the slow path together
@@ -434,7 +452,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 m_ref = m_new;
             }
             // p = 2^(c*s - m_ref); row sum from the fp32 values; P packed to bf16 over the first 64 columns of S
-            float psum = 0.f;
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial row sums
             if constexpr (!kLowReg) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -442,7 +460,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     for (int i = 0; i < 32; i += 2) {
                         const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_ref));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_ref));
-                        psum += p0 + p1;
+                        ps[(i >> 1) & 3] += p0 + p1;
                         sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
                     }
                 }
@@ -465,14 +483,14 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                             if (c * 32 + i >= valid) p0 = 0.f;
                             if (c * 32 + i + 1 >= valid) p1 = 0.f;
                         }
-                        psum += p0 + p1;
+                        ps[(i >> 1) & 3] += p0 + p1;
                         pk[i / 2] = pack_bf16(p0, p1);
                     }
                     tmem_wait_ld();            // chunk c+1 has landed before P overwrites columns below it
                     tmem_st16(s_addr + c * 16, pk);
                 }
             }
-            l_sum += psum;
+            l_sum += (ps[0] + ps[1]) + (ps[2] + ps[3]);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p(b));
@@ -536,31 +554,31 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 template <int D>
 __global__ void __launch_bounds__(320, 1)
 prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
                   float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
 }
 
-// 152 registers per thread: two of these warps and one suffix warp (208) fill the 512 registers per lane of
+// At most 144 registers per thread: two of these warps and one suffix warp (208) fit the 512 registers per lane of
 // an SM sub-partition, which is what lets a suffix block run beside this block.
 template <int D>
-__global__ void __maxnreg__(152)
+__global__ void __maxnreg__(144)
 prefix_kernel_one(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
                   float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
 }
 
 // One row tile, long items: the block owns the SM anyway (long ring), so S stays in registers.
 template <int D>
 __global__ void __launch_bounds__(192, 1)
 prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int ring,
+                       const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
                        float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, ring, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
 }
 
 // ---------------------------------------------------------------- host side
@@ -597,7 +615,8 @@ bool encode(EncodeFn fn, CUtensorMap *map, const void *base, int rank, const cuu
     return true;
 }
 
-// kShape: 2 = two row tiles, 1 = one row tile with short items (small block), 0 = one row tile with long items
+// kShape: 2 = two row tiles; 1 = one row tile, small block that can share the SM with a suffix block (short items,
+// or enough rows per tile that the block is not purely HBM-bound); 0 = one row tile, long ring, owns the SM
 template <int D, int kShape>
 int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
 {
@@ -606,13 +625,11 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     auto kern = kShape == 2 ? prefix_kernel_two<D> : (kShape == 1 ? prefix_kernel_one<D> : prefix_kernel_one_long<D>);
     // ring length: enough buffers for the epilogue staging tile(s); short items of the one-row-tile
     // shape get the smallest block so that a suffix block fits beside it on the SM
-    constexpr int kLongRing = (kTwo && D == 128) ? 5 : kMaxRing;   // the longest ring that fits in 227 KB
-    static_assert(L::total(kLongRing) <= 227 * 1024 && L::min_ring() <= kLongRing, "shared memory plan does not fit");
-    int ring = kShape == 1 ? 3 : kLongRing;
-    ring = ring < L::min_ring() ? L::min_ring() : ring;
+    constexpr int ring = prefix_ring<D, kTwo, kShape == 1>();
+    static_assert(L::total(ring) <= 227 * 1024 && L::min_ring() <= ring, "shared memory plan does not fit");
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total(kLongRing));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total(ring));
         if (e != cudaSuccess) return int(e);
         // ask for the largest shared-memory carve-out so that a suffix block can share the SM
         e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -620,7 +637,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
         configured = true;
     }
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
-    kern<<<a.num_items, kTwo ? 320 : 192, L::total(ring), st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, ring,
+    kern<<<a.num_items, kTwo ? 320 : 192, L::total(ring), st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads,
                                                                scale_log2, a.partial_o, a.partial_lse, a.status);
     return int(cudaGetLastError());
 }
@@ -651,7 +668,7 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc;
     if (a.max_rows_per_item > kPrefixTileRows) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
-    else if (a.max_tiles_per_item <= 2) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
+    else if (a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
     else rc = D == 128 ? launch_one<128, 0>(a, mq, mk, mv, st) : launch_one<64, 0>(a, mq, mk, mv, st);
     if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));
     return rc;
