@@ -28,7 +28,25 @@ import psa_workloads as wl  # noqa: E402
 METRIC = "sample-tokens/sec per decode step"
 UNIT = "sample-tokens/s"
 L2_BYTES = 126e6
+# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu launch list of this very command
+# (profiles/launch_list_bench_cfg2.md).  Only valid for the kernel source it was taken with.
+NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68270655 + 16007,
+                        "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "93c285341b3d3d1f"}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def ncu_traffic(config_name):
+    import hashlib
+    t = NCU_TRAFFIC.get(config_name)
+    if not t:
+        return None
+    try:
+        with open(os.path.join(ROOT, t["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != t["sha256_16"]:
+                return None          # the kernel changed since the counters were taken
+    except OSError:
+        return None
+    return t["bytes_per_launch"]
 
 
 def load_peaks():
@@ -195,7 +213,13 @@ def run_psa(args, cfg):
                 fn(i)
         return g
 
-    graphs = [capture(lambda _, i=i: step(i), 1) for i in range(n_copies)]
+    # one graph holds `per_graph` consecutive steps (one per input copy); a second one holds the remainder,
+    # so that exactly args.steps steps are timed
+    per_graph = max(n_copies, 8) if args.steps >= 8 else 1
+    g_full = capture(step, per_graph)
+    per_graph_steps = per_graph
+    n_full, n_rest = divmod(args.steps, per_graph)
+    g_rest = capture(step, n_rest) if n_rest else None
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def timed(run_one, steps, warmup):
@@ -209,15 +233,25 @@ def run_psa(args, cfg):
         barrier()
         return ev0.elapsed_time(ev1)
 
-    ms_total = timed(lambda i: graphs[i % n_copies].replay(), args.steps, args.warmup)
+    for _ in range(-(-args.warmup // per_graph)):
+        g_full.replay()
+    barrier()
+    ev0.record()
+    for _ in range(n_full):
+        g_full.replay()
+    if g_rest is not None:
+        g_rest.replay()
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
     plan.check_status()
     eager_steps = min(args.steps, 500)
     ms_eager = timed(step, eager_steps, min(args.warmup, 10)) / eager_steps
 
     # ---- per-stage durations: each stage alone, launched back to back over the same rotating copies
     stage_avg = {}
+    reps = max(1, min(args.steps, 400) // max(n_copies, 8))
     per_graph = max(n_copies, 8)
-    reps = max(1, min(args.steps, 400) // per_graph)
     for name in ("prefix", "suffix", "merge"):
         g = capture(lambda i, name=name: step(i, name), per_graph)
         stage_avg[name] = timed(lambda i: g.replay(), reps, 2) / (reps * per_graph)
@@ -285,7 +319,7 @@ def run_psa(args, cfg):
                        "kv_heads": w["num_kv_heads"], "head_dim": D, "prefix_len": list(cfg.prefix_len),
                        "suffix_len": list(cfg.suffix_len), "page_size": 16,
                        "cold_l2": f"steps rotate over {n_copies} input copies ({n_copies * input_bytes / 1e6:.0f} MB > L2 126 MB)",
-                       "launch": "CUDA graph replay, one captured psa_decode per step",
+                       "launch": f"CUDA graph replay, {per_graph_steps} captured psa_decode steps per graph",
                        "sharding": "independent prompts per rank, no collective"},
             "plan": {"prefix_items": info.num_prefix_items, "suffix_items": info.num_suffix_items,
                      "prefix_tiles_per_item": info.prefix_tiles_per_item, "suffix_chunk_tokens": info.suffix_chunk_tokens},
@@ -293,7 +327,7 @@ def run_psa(args, cfg):
             "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps, "entry_point": "psa_decode_host"},
             "roofline": {"kernel": "suffix_kernel", "bound": "hbm", "achieved": suf_gbs, "peak": hbm, "unit": "GB/s",
-                         "frac": suf_gbs / hbm if suf_gbs else None, "traffic": None, "peak_kind": f"of {peaks_kind}",
+                         "frac": suf_gbs / hbm if suf_gbs else None, "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peaks_kind}",
                          "algorithmic_bytes_per_launch": abytes["suffix"]},
             "kernels": kernels,
             "eager_ms_per_step": ms_eager,

@@ -155,14 +155,14 @@ def make_workload(cfg: PsaConfig, poison: bool = False, lengths=None) -> dict:
 
 def checksum(w: dict) -> int:
     """Order-sensitive 64-bit checksum of the tensors, to tell runs apart in logs."""
-    acc = np.uint64(1469598103934665603)
+    acc = 1469598103934665603
     for name in ("q", "prefix_k", "prefix_v", "pool_k", "pool_v", "page_indices", "suffix_lens"):
         a = np.ascontiguousarray(w[name]).view(np.uint8)
         pad = (-a.size) % 8
         if pad:
             a = np.concatenate([a.ravel(), np.zeros(pad, np.uint8)])
-        acc = acc * np.uint64(1099511628211) + np.bitwise_xor.reduce(a.ravel().view(np.uint64), dtype=np.uint64)
-    return int(acc)
+        acc = (acc * 1099511628211 + int(np.bitwise_xor.reduce(a.ravel().view(np.uint64)))) & 0xFFFFFFFFFFFFFFFF
+    return acc
 
 
 def algorithmic_bytes(w: dict) -> dict:
