@@ -27,6 +27,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
              void *__restrict__ out, float *__restrict__ lse_out)
 {
     constexpr int V = D / 32;  // floats per lane: 2 or 4
+    constexpr int kChunk = 8;  // rows fetched together (registers: kChunk float4 per lane)
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
     if (row >= num_rows) return;
@@ -51,63 +52,60 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // pass 1: the largest lse (lanes stride over the partials)
-    float top = -INFINITY;
-    for (int i = lane; i < n_total; i += 32) top = fmaxf(top, __ldcg(partial_lse + partial_row(i)));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, o));
-
-    // pass 2: lane i of each group of 32 partials computes weight and row; the rows are then
-    // fetched eight at a time so that several loads are in flight per lane
+    // Single pass with a running maximum (the same deferred-division bookkeeping as inside the kernels):
+    // per group of 32 partials, lane i loads lse_i while the first kChunk output rows of the group are already
+    // being fetched -- row addresses do not depend on the lse values -- so the lse round trip
+    // and the first row round trip overlap.
     float acc[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = 0.f;
-    float z = 0.f;
+    float top = -INFINITY, z = 0.f;   // z: this lane's share of sum_i exp(lse_i - top)
     auto fetch = [&](int r) {
         const float *src = partial_o + size_t(r) * D + lane * V;
         if constexpr (V == 4) return __ldcg(reinterpret_cast<const float4 *>(src));
         else { const float2 x = __ldcg(reinterpret_cast<const float2 *>(src)); return make_float4(x.x, x.y, 0.f, 0.f); }
     };
-    auto fma_row = [&](float w, const float4 &x) {
-        acc[0] += w * x.x; acc[1] += w * x.y;
-        if constexpr (V == 4) { acc[2] += w * x.z; acc[3] += w * x.w; }
-    };
-    if (top != -INFINITY) {
-        for (int base = 0; base < n_total; base += 32) {
-            const int mine = base + lane;
-            const int my_row = mine < n_total ? partial_row(mine) : 0;
-            // an empty piece (lse = -inf) gets weight 0
-            const float my_w = mine < n_total ? __expf(__ldcg(partial_lse + my_row) - top) : 0.f;
-            z += my_w;
-            const int cnt = min(32, n_total - base);
-            int i = 0;
-            for (; i + 8 <= cnt; i += 8) {
-                float4 x[8]; float w[8];
+    for (int base = 0; base < n_total; base += 32) {
+        const int mine = base + lane;
+        const int my_row = mine < n_total ? partial_row(mine) : 0;
+        const float my_lse = mine < n_total ? __ldcg(partial_lse + my_row) : -INFINITY;
+        const int cnt = min(32, n_total - base);
+        float my_w = 0.f;
+        for (int c0 = 0; c0 < cnt; c0 += kChunk) {
+            float4 x[kChunk];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    w[u] = __shfl_sync(0xffffffffu, my_w, i + u);
-                    x[u] = fetch(__shfl_sync(0xffffffffu, my_row, i + u));
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) fma_row(w[u], x[u]);
+            for (int u = 0; u < kChunk; ++u) {
+                const int r = __shfl_sync(0xffffffffu, my_row, (c0 + u) & 31);
+                x[u] = (c0 + u < cnt) ? fetch(r) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            for (; i + 2 <= cnt; i += 2) {
-                float4 x[2]; float w[2];
+            if (c0 == 0) {   // first use of the lse values of this group
+                float gmax = my_lse;
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    w[u] = __shfl_sync(0xffffffffu, my_w, i + u);
-                    x[u] = fetch(__shfl_sync(0xffffffffu, my_row, i + u));
+                for (int o = 16; o > 0; o >>= 1) gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
+                const float new_top = fmaxf(top, gmax);
+                if (new_top != -INFINITY) {
+                    const float scale = __expf(top - new_top);   // 0 when nothing was accumulated yet
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc[v] *= scale;
+                    z *= scale;
+                    top = new_top;
+                    my_w = __expf(my_lse - top);                 // an empty piece (lse = -inf) gets weight 0
+                    z += my_w;
                 }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) fma_row(w[u], x[u]);
             }
-            for (; i < cnt; ++i) {
-                const float w = __shfl_sync(0xffffffffu, my_w, i);
-                fma_row(w, fetch(__shfl_sync(0xffffffffu, my_row, i)));
+#pragma unroll
+            for (int u = 0; u < kChunk; ++u) {
+                const float w = __shfl_sync(0xffffffffu, my_w, (c0 + u) & 31);
+                if (c0 + u < cnt) {
+                    acc[0] += w * x[u].x; acc[1] += w * x[u].y;
+                    if constexpr (V == 4) { acc[2] += w * x[u].z; acc[3] += w * x[u].w; }
+                }
             }
         }
+    }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    if (top != -INFINITY) {
         const float inv = 1.f / z;
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] *= inv;

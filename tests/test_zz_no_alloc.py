@@ -47,16 +47,16 @@ def test_static_workspace_matches_decode_on_two_calls_in_a_row():
 
 
 def test_static_workspace_rejects_plans_beyond_its_size():
-    from paper_2502_02534_b200 import PsaError, decode_static
-    from paper_2502_02534_b200.binding import STATIC_WORKSPACE_BYTES
-    w = wl.make_workload(wl.CONFIGS["cfg3"])          # needs ~21.6 MB of workspace
-    plan = make_plan(w, "bf16")
-    assert plan.workspace_bytes > STATIC_WORKSPACE_BYTES
-    dev = to_device(w)
     import torch
-    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
-    out = torch.zeros((B, Hq, D), dtype=torch.bfloat16, device="cuda"); lse = torch.zeros((B, Hq), dtype=torch.float32, device="cuda")
+    from paper_2502_02534_b200 import Plan, PsaError, decode_static
+    from paper_2502_02534_b200.binding import STATIC_WORKSPACE_BYTES
+    cfg = wl.CONFIGS["cfg4"]                           # 256 samples x 64 heads: ~30 MB of partial results
+    L, N, S = wl.draw_lengths(cfg)                     # lengths only: the size check comes before any memory access
+    plan = Plan(L, N, S, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads, head_dim=cfg.head_dim)
+    assert plan.workspace_bytes > STATIC_WORKSPACE_BYTES
+    dummy = torch.zeros(1024, dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros(1024, dtype=torch.int32, device="cuda")
+    lse = torch.zeros(1024, dtype=torch.float32, device="cuda")
     with pytest.raises(PsaError) as e:
-        decode_static(plan, dev["q"], dev["prefix_k"], dev["prefix_v"], dev["pool_k"], dev["pool_v"], dev["page_indptr"],
-                      dev["page_indices"], dev["suffix_lens"], out, lse)
+        decode_static(plan, dummy, dummy, dummy, dummy, dummy, idx, idx, idx, dummy, lse)
     assert e.value.status == 3 and "PSA_STATIC_WORKSPACE_BYTES" in str(e.value)
