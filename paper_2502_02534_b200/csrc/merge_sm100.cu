@@ -19,7 +19,7 @@ namespace {
 
 constexpr int kMergeWarps = 4;
 
-template <int D>
+template <int D, int kChunk>
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restrict__ suffix_lens,
              const float *__restrict__ partial_o, const float *__restrict__ partial_lse,
@@ -27,7 +27,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
              void *__restrict__ out, float *__restrict__ lse_out)
 {
     constexpr int V = D / 32;  // floats per lane: 2 or 4
-    constexpr int kChunk = 8;  // rows fetched together (registers: kChunk float4 per lane)
+    // kChunk rows are fetched together (registers: kChunk float4 per lane)
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
     if (row >= num_rows) return;
@@ -51,6 +51,9 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
 
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the next kernel in the stream (typically the next step's prefix stage) may set itself up meanwhile;
+    // it waits for this grid to complete before it touches memory
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // Single pass with a running maximum (the same deferred-division bookkeeping as inside the kernels):
     // per group of 32 partials, lane i loads lse_i while the first kChunk output rows of the group are already
@@ -150,11 +153,15 @@ int launch_merge(const MergeArgs &a, void *stream, std::string *err)
     lc.numAttrs = a.after_stage ? 1 : 0;   // start filling in while the preceding stage drains
     const int f32 = a.out_dtype == PSA_OUT_F32;
     cudaError_t e;
-    if (a.head_dim == 128)
-        e = cudaLaunchKernelEx(&lc, merge_kernel<128>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+    const bool small = rows <= 4096;   // few rows: latency matters, fetch 16 partial rows at a time
+    if (a.head_dim == 128 && small)
+        e = cudaLaunchKernelEx(&lc, merge_kernel<128, 16>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
+    else if (a.head_dim == 128)
+        e = cudaLaunchKernelEx(&lc, merge_kernel<128, 8>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
                                a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
     else
-        e = cudaLaunchKernelEx(&lc, merge_kernel<64>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+        e = cudaLaunchKernelEx(&lc, merge_kernel<64, 16>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
                                a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
     if (e != cudaSuccess && err) *err = std::string("merge launch: ") + cudaGetErrorString(e);
     return int(e);

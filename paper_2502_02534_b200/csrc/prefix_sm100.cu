@@ -279,7 +279,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
-    // every block is resident now: a kernel launched as a programmatic dependent may start filling the machine
+    // Launched as a programmatic dependent of whatever precedes it in the stream, this block did its set-up
+    // while that kernel drained; from here on it reads inputs and (later) overwrites partial results, so the
+    // predecessor must be complete.  Only then may our own dependent (the suffix stage) start beside us.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kProducerWarp) {
@@ -637,9 +640,18 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
         configured = true;
     }
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
-    kern<<<a.num_items, kTwo ? 320 : 192, L::total(ring), st>>>(mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads,
-                                                               scale_log2, a.partial_o, a.partial_lse, a.status);
-    return int(cudaGetLastError());
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(a.num_items);
+    lc.blockDim = dim3(kTwo ? 320 : 192);
+    lc.dynamicSmemBytes = L::total(ring);
+    lc.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = 1;   // set-up may overlap the tail of the preceding kernel; the kernel waits before touching memory
+    return int(cudaLaunchKernelEx(&lc, kern, mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, scale_log2, a.partial_o,
+                                  a.partial_lse, a.status));
 }
 
 }  // namespace
