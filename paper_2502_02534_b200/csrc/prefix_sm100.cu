@@ -213,7 +213,7 @@ struct PrefixSmem {
     static constexpr int kRingOff = kQOff + kQTiles * kTileBytes;
     static constexpr int kStageRowFloats = D + 4;                     // padded row of the epilogue staging tile
     static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;
-    static constexpr int kTmemCols = 512;                             // S0 S1 (128 each) at 0, O0 O1 (D each) at 256
+    static constexpr int kTmemCols = 512;   // S0 S1 (128 each) at 0; O0 O1 (D each) at 256, or O at 256 and P0 P1 at 384
     __host__ __device__ static constexpr int total(int ring) { return kRingOff + ring * kTileBytes; }
     __host__ __device__ static constexpr int min_ring() { return (kQTiles * kStageBytes + kTileBytes - 1) / kTileBytes; }
 };
@@ -233,6 +233,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     constexpr uint32_t kIdescQK = make_idesc(kPrefixTileKeys, false);
     constexpr uint32_t kIdescPV = make_idesc(D, true);
     constexpr uint32_t kColS = 0, kColO = 2 * kPrefixTileKeys;
+    constexpr uint32_t kColP = 384;   // one row tile only: P0, P1 (64 columns each) behind O
 
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -321,7 +322,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             };
             auto issue_pv = [&](int t, int j) {   // O_t += P[sbuf] V_j ; V_j is ring entry 2j+1
                 const uint32_t vb = sbase + L::kRingOff + ((2 * j + 1) % ring) * L::kTileBytes;
-                const uint32_t a = tmem_base + kColS + sbuf(t, j) * kPrefixTileKeys;
+                const uint32_t a = kTwo ? tmem_base + kColS + t * kPrefixTileKeys   // P over S
+                                        : tmem_base + kColP + (j & 1) * (kPrefixTileKeys / 2);
 #pragma unroll
                 for (int k = 0; k < kPSteps; ++k)
                     mma_ts(tmem_base + kColO + t * D, a + k * 8, make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV,
@@ -389,8 +391,35 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             if (!(ok = mbar_wait(bar_s(b), sphase(j), abort_flag))) break;
             tc_fence_after();
             const int valid = n_keys - j * kPrefixTileKeys;   // >= 1; < 128 only on the last tile
-            float tmax = -INFINITY;
-            if constexpr (!kLowReg) {
+
+            // Rescale the accumulator in TMEM by 2^(m_ref - m_new) for the rows whose reference maximum moves.
+            // The whole warp comes here together because TMEM loads and stores are warp-collective.
+            auto move_reference = [&](bool need, float m_new) -> bool {
+                const float alpha = need ? fast_exp2(m_ref - m_new) : 1.f;   // 0 on the first tile
+                if (j > 0) {
+                    // O must be quiescent: PV of tile j-1 has to be complete, which is what releases the ring
+                    // buffer of V_{j-1} (PV of tile j cannot start before this thread hands over P)
+                    if (!mbar_wait(bar_empty((2 * j - 1) % ring), ((2 * j - 1) / ring) & 1, abort_flag)) return false;
+                    tc_fence_after();
+                    uint32_t oreg[32];
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(o_addr + c * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
+                        tmem_st32(o_addr + c * 32, oreg);
+                    }
+                    tmem_wait_st();
+                }
+                l_sum *= alpha;
+                if (need) m_ref = m_new;
+                return true;
+            };
+
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial row sums
+            if constexpr (kTwo) {
+                // ---- S in registers; P (bf16) is written back over the first 64 columns of S
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
                 tmem_wait_ld();
@@ -406,57 +435,12 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(sreg[c][i]));   // eight independent chains
-                tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-            } else {
-                // low-register form: S is read twice from TMEM, 32 columns at a time (pass 1: maximum)
-                uint32_t r[2][32];
-                float mx[2] = {-INFINITY, -INFINITY};
-                tmem_ld32(s_addr, r[0]);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
-                    if (valid >= kPrefixTileKeys) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c * 32 + i < valid) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
-                    }
-                    tmem_wait_ld();
+                const float tmax = scale_log2 * fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                // move the reference maximum only when a logit exceeds it by more than the threshold
+                const bool need = tmax > m_ref + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    if (!(ok = move_reference(need, tmax))) break;
                 }
-                tmax = fmaxf(mx[0], mx[1]);
-            }
-            tmax *= scale_log2;
-            // Move the reference maximum only when needed; the whole warp takes the slow path together
-            // because TMEM loads and stores are warp-collective.
-            const bool need = tmax > m_ref + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {
-                const float m_new = need ? tmax : m_ref;
-                const float alpha = need ? fast_exp2(m_ref - m_new) : 1.f;   // 0 on the first tile
-                if (j > 0) {
-                    // O must be quiescent: PV of tile j-1 has to be complete, which is what releases the ring
-                    // buffer of V_{j-1} (PV of tile j cannot start before this thread hands over P)
-                    if (!(ok = mbar_wait(bar_empty((2 * j - 1) % ring), ((2 * j - 1) / ring) & 1, abort_flag))) break;
-                    tc_fence_after();
-                    uint32_t oreg[32];
-#pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
-                        tmem_ld32(o_addr + c * 32, oreg);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
-                        tmem_st32(o_addr + c * 32, oreg);
-                    }
-                    tmem_wait_st();
-                }
-                l_sum *= alpha;
-                m_ref = m_new;
-            }
-            // p = 2^(c*s - m_ref); row sum from the fp32 values; P packed to bf16 over the first 64 columns of S
-            float ps[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial row sums
-            if constexpr (!kLowReg) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
 #pragma unroll
@@ -470,27 +454,65 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 tmem_st32(s_addr, sreg[0]);
                 tmem_st32(s_addr + 32, sreg[1]);
             } else {
-                // pass 2: chunk c of S (columns 32c..32c+31) becomes columns 16c..16c+15 of P, which were read already
-                uint32_t r[2][32];
-                tmem_ld32(s_addr, r[0]);
-                tmem_wait_ld();
+                // ---- one row tile: P has TMEM columns of its own, so S stays intact and the common case is a
+                // single pass that exponentiates against the CURRENT reference maximum while tracking the
+                // largest exponent; only if that exceeds the threshold (or on the first tile) is the tile redone
+                // after moving the reference.  S is streamed 32 columns at a time (two chunks in flight).
+                const uint32_t p_addr = tmem_base + lane_addr + kColP + b * (kPrefixTileKeys / 2);
+                auto exp_pass = [&](float &xmax) {
+                    uint32_t r[2][32];
+                    float mx[2] = {-INFINITY, -INFINITY};
+                    ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
+                    tmem_ld32(s_addr, r[0]);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
-                    uint32_t pk[16];
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+                        uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_ref));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_ref));
-                        if (valid < kPrefixTileKeys) {
-                            if (c * 32 + i >= valid) p0 = 0.f;
-                            if (c * 32 + i + 1 >= valid) p1 = 0.f;
+                        for (int i = 0; i < 32; i += 2) {
+                            float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_ref);
+                            float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_ref);
+                            if (valid < kPrefixTileKeys) {   // masked keys of a ragged last tile
+                                if (c * 32 + i >= valid) x0 = -INFINITY;
+                                if (c * 32 + i + 1 >= valid) x1 = -INFINITY;
+                            }
+                            mx[0] = fmaxf(mx[0], x0);
+                            mx[1] = fmaxf(mx[1], x1);
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                            ps[(i >> 1) & 3] += p0 + p1;
+                            pk[i / 2] = pack_bf16(p0, p1);
                         }
-                        ps[(i >> 1) & 3] += p0 + p1;
-                        pk[i / 2] = pack_bf16(p0, p1);
+                        tmem_st16(p_addr + c * 16, pk);
+                        tmem_wait_ld();
                     }
-                    tmem_wait_ld();            // chunk c+1 has landed before P overwrites columns below it
-                    tmem_st16(s_addr + c * 16, pk);
+                    xmax = fmaxf(mx[0], mx[1]);
+                };
+                bool redo = j == 0;   // nothing to exponentiate against yet
+                if (j > 0) {
+                    float xmax;
+                    exp_pass(xmax);
+                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold);
+                }
+                if (redo) {
+                    // the tile's maximum, then the classic update, then the exponentials again
+                    uint32_t r[2][32];
+                    float mx[2] = {-INFINITY, -INFINITY};
+                    tmem_ld32(s_addr, r[0]);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (valid >= kPrefixTileKeys || c * 32 + i < valid) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
+                        tmem_wait_ld();
+                    }
+                    const float tmax = scale_log2 * fmaxf(mx[0], mx[1]);
+                    const bool need = tmax > m_ref + kRescaleThreshold;
+                    if (!(ok = move_reference(need, tmax))) break;
+                    float xmax;
+                    exp_pass(xmax);
                 }
             }
             l_sum += (ps[0] + ps[1]) + (ps[2] + ps[3]);
