@@ -195,22 +195,28 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 // Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 10 warps); otherwise one row
 // tile (one Q tile, 6 warps).
 constexpr int kMaxRing = 6;
-// Ring length per block shape: 5 x 32 KB beside two Q tiles, 6 when the block owns the SM, 3 for the small
-// block that shares the SM with a suffix block (never fewer buffers than the epilogue staging tile needs).
+// Ring length per block shape: 5 x 32 KB beside two Q tiles, else 6 (never fewer buffers than the epilogue
+// staging tile needs).
 template <int D, bool kTwo, bool kLowReg>
-__host__ __device__ constexpr int prefix_ring() { return kLowReg ? 3 : ((kTwo && D == 128) ? 5 : kMaxRing); }
-template <int D, bool kTwo>
+__host__ __device__ constexpr int prefix_ring() { return (kTwo && D == 128) ? 5 : kMaxRing; }
+// Keys per tile: 128, except in the small block, whose 96 KB ring then holds six 64-key tiles (three tiles of
+// look-ahead) instead of three 128-key tiles (none: every load would wait for the previous tile's MMA).
+template <bool kLowReg>
+__host__ __device__ constexpr int prefix_tile_keys() { return kLowReg ? 64 : kPrefixTileKeys; }
+template <int D, bool kTwo, int kKeys>
 struct PrefixSmem {
-    static constexpr int kHalfBytes = kPrefixTileKeys * 128;          // one TMA box: 128 rows x 64 bf16
     static constexpr int kHalves = D / 64;
-    static constexpr int kTileBytes = kHalves * kHalfBytes;           // a Q, K or V tile
+    static constexpr int kQHalfBytes = kPrefixTileRows * 128;         // one TMA box of Q: 128 rows x 64 bf16
+    static constexpr int kQTileBytes = kHalves * kQHalfBytes;
+    static constexpr int kHalfBytes = kKeys * 128;                    // one TMA box of K or V: kKeys rows x 64 bf16
+    static constexpr int kTileBytes = kHalves * kHalfBytes;           // a K or V tile
     static constexpr int kQTiles = kTwo ? 2 : 1;
     static constexpr int kBarOff = 0;                                 // barriers first, tiles after them
     static constexpr int kNumBars = 1 + 2 * kMaxRing + 4;             // q, full[], empty[], s_full[2], p_full[2]
     static constexpr int kTmemPtrOff = kBarOff + 8 * kNumBars;
     static constexpr int kAbortOff = kTmemPtrOff + 4;
     static constexpr int kQOff = 1024;
-    static constexpr int kRingOff = kQOff + kQTiles * kTileBytes;
+    static constexpr int kRingOff = kQOff + kQTiles * kQTileBytes;
     static constexpr int kStageRowFloats = D + 4;                     // padded row of the epilogue staging tile
     static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;
     static constexpr int kTmemCols = 512;   // S0 S1 (128 each) at 0; O0 O1 (D each) at 256, or O at 256 and P0 P1 at 384
@@ -224,15 +230,17 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             const PrefixItem *__restrict__ items, int group, float scale_log2,
             float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    using L = PrefixSmem<D, kTwo>;
+    constexpr int kKeys = prefix_tile_keys<kLowReg>();   // keys per tile
+    using L = PrefixSmem<D, kTwo, kKeys>;
     constexpr int ring = prefix_ring<D, kTwo, kLowReg>();   // K/V tile buffers in flight
     constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
     constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
     constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
-    constexpr int kPSteps = kPrefixTileKeys / 16;   // MMA k-steps of PV
-    constexpr uint32_t kIdescQK = make_idesc(kPrefixTileKeys, false);
+    constexpr int kPSteps = kKeys / 16;   // MMA k-steps of PV
+    constexpr uint32_t kIdescQK = make_idesc(kKeys, false);
     constexpr uint32_t kIdescPV = make_idesc(D, true);
-    constexpr uint32_t kColS = 0, kColO = 2 * kPrefixTileKeys;
+    constexpr uint32_t kColS = 0, kColO = 256;   // S buffer b at column 128 b (kKeys of them in use)
+    constexpr int kChunks = kKeys / 32;          // 32-column pieces of one S tile
     constexpr uint32_t kColP = 384;   // one row tile only: P0, P1 (64 columns each) behind O
 
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -255,7 +263,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     const int4 it1 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x) + 1);
     const int first_token = it0.x, n_keys = it0.y, kv = it0.z, first_sample = it0.w;
     const int n_rows = it1.x, prow0 = it1.y;
-    const int n_tiles = (n_keys + kPrefixTileKeys - 1) / kPrefixTileKeys;
+    const int n_tiles = (n_keys + kKeys - 1) / kKeys;
     const int n_rt = kTwo ? (n_rows > kPrefixTileRows ? 2 : 1) : 1;   // row tiles in use
     const int samples_per_tile = kPrefixTileRows / group;
 
@@ -289,16 +297,16 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            mbar_expect_tx(bar_q(), n_rt * L::kTileBytes);
+            mbar_expect_tx(bar_q(), n_rt * L::kQTileBytes);
             for (int t = 0; t < n_rt; ++t)
                 for (int h = 0; h < L::kHalves; ++h)
-                    tma_load_4d(sbase + L::kQOff + t * L::kTileBytes + h * L::kHalfBytes, pmap_q, bar_q(), h * 64, 0, kv,
+                    tma_load_4d(sbase + L::kQOff + t * L::kQTileBytes + h * L::kQHalfBytes, pmap_q, bar_q(), h * 64, 0, kv,
                                 first_sample + t * samples_per_tile);
             // ring order: K0 V0 K1 V1 ...
             for (int i = 0; i < 2 * n_tiles; ++i) {
                 const int slot = i % ring, use = i / ring;
                 if (use > 0 && !mbar_wait(bar_empty(slot), (use - 1) & 1, abort_flag)) break;
-                const int tok = first_token + (i >> 1) * kPrefixTileKeys;
+                const int tok = first_token + (i >> 1) * kKeys;
                 const CUtensorMap *map = (i & 1) ? pmap_v : pmap_k;
                 mbar_expect_tx(bar_full(slot), L::kTileBytes);
                 for (int h = 0; h < L::kHalves; ++h)
@@ -311,19 +319,19 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             bool ok = mbar_wait(bar_q(), 0, abort_flag);
             auto wait_entry = [&](int e) { return mbar_wait(bar_full(e % ring), (e / ring) & 1, abort_flag); };
             auto issue_qk = [&](int t, int j) {   // S[sbuf] = Q_t K_j^T ; K_j is ring entry 2j
-                const uint32_t qa = sbase + L::kQOff + t * L::kTileBytes;
+                const uint32_t qa = sbase + L::kQOff + t * L::kQTileBytes;
                 const uint32_t kb = sbase + L::kRingOff + ((2 * j) % ring) * L::kTileBytes;
-                const uint32_t d = tmem_base + kColS + sbuf(t, j) * kPrefixTileKeys;
+                const uint32_t d = tmem_base + kColS + sbuf(t, j) * 128;
 #pragma unroll
                 for (int k = 0; k < kKSteps; ++k) {
-                    const uint32_t off = (k / 4) * L::kHalfBytes + (k % 4) * 32;
-                    mma_ss(d, make_smem_desc(qa + off, 16, 1024), make_smem_desc(kb + off, 16, 1024), kIdescQK, k > 0);
+                    mma_ss(d, make_smem_desc(qa + (k / 4) * L::kQHalfBytes + (k % 4) * 32, 16, 1024),
+                           make_smem_desc(kb + (k / 4) * L::kHalfBytes + (k % 4) * 32, 16, 1024), kIdescQK, k > 0);
                 }
             };
             auto issue_pv = [&](int t, int j) {   // O_t += P[sbuf] V_j ; V_j is ring entry 2j+1
                 const uint32_t vb = sbase + L::kRingOff + ((2 * j + 1) % ring) * L::kTileBytes;
-                const uint32_t a = kTwo ? tmem_base + kColS + t * kPrefixTileKeys   // P over S
-                                        : tmem_base + kColP + (j & 1) * (kPrefixTileKeys / 2);
+                const uint32_t a = kTwo ? tmem_base + kColS + t * 128   // P over S
+                                        : tmem_base + kColP + (j & 1) * 64;
 #pragma unroll
                 for (int k = 0; k < kPSteps; ++k)
                     mma_ts(tmem_base + kColO + t * D, a + k * 8, make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV,
@@ -387,10 +395,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         uint32_t sreg[4][32];
         for (int j = 0; j < n_tiles; ++j) {
             const int b = sbuf(t, j);
-            const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kPrefixTileKeys;
+            const uint32_t s_addr = tmem_base + lane_addr + kColS + b * 128;
             if (!(ok = mbar_wait(bar_s(b), sphase(j), abort_flag))) break;
             tc_fence_after();
-            const int valid = n_keys - j * kPrefixTileKeys;   // >= 1; < 128 only on the last tile
+            const int valid = n_keys - j * kKeys;   // >= 1; < kKeys only on the last tile
 
             // Rescale the accumulator in TMEM by 2^(m_ref - m_new) for the rows whose reference maximum moves.
             // The whole warp comes here together because TMEM loads and stores are warp-collective.
@@ -424,7 +432,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
                 tmem_wait_ld();
                 float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (valid < kPrefixTileKeys) {   // last tile of a ragged prompt: masked keys become -inf
+                if (valid < kKeys) {   // last tile of a ragged prompt: masked keys become -inf
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -458,7 +466,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 // single pass that exponentiates against the CURRENT reference maximum while tracking the
                 // largest exponent; only if that exceeds the threshold (or on the first tile) is the tile redone
                 // after moving the reference.  S is streamed 32 columns at a time (two chunks in flight).
-                const uint32_t p_addr = tmem_base + lane_addr + kColP + b * (kPrefixTileKeys / 2);
+                const uint32_t p_addr = tmem_base + lane_addr + kColP + b * 64;
                 auto exp_pass = [&](float &xmax) {
                     uint32_t r[2][32];
                     float mx[2] = {-INFINITY, -INFINITY};
@@ -466,14 +474,14 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     tmem_ld32(s_addr, r[0]);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+                    for (int c = 0; c < kChunks; ++c) {
+                        if (c + 1 < kChunks) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
                             float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_ref);
                             float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_ref);
-                            if (valid < kPrefixTileKeys) {   // masked keys of a ragged last tile
+                            if (valid < kKeys) {   // masked keys of a ragged last tile
                                 if (c * 32 + i >= valid) x0 = -INFINITY;
                                 if (c * 32 + i + 1 >= valid) x1 = -INFINITY;
                             }
@@ -501,11 +509,11 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     tmem_ld32(s_addr, r[0]);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < 3) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
+                    for (int c = 0; c < kChunks; ++c) {
+                        if (c + 1 < kChunks) tmem_ld32(s_addr + (c + 1) * 32, r[(c + 1) & 1]);
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
-                            if (valid >= kPrefixTileKeys || c * 32 + i < valid) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
+                            if (valid >= kKeys || c * 32 + i < valid) mx[i & 1] = fmaxf(mx[i & 1], __uint_as_float(r[c & 1][i]));
                         tmem_wait_ld();
                     }
                     const float tmax = scale_log2 * fmaxf(mx[0], mx[1]);
@@ -646,7 +654,7 @@ template <int D, int kShape>
 int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
 {
     constexpr bool kTwo = kShape == 2;
-    using L = PrefixSmem<D, kTwo>;
+    using L = PrefixSmem<D, kTwo, prefix_tile_keys<kShape == 1>()>;
     auto kern = kShape == 2 ? prefix_kernel_two<D> : (kShape == 1 ? prefix_kernel_one<D> : prefix_kernel_one_long<D>);
     // ring length: enough buffers for the epilogue staging tile(s); short items of the one-row-tile
     // shape get the smallest block so that a suffix block fits beside it on the SM
@@ -685,6 +693,9 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     if (!fn) return int(cudaErrorNotSupported);
     const int G = a.num_q_heads / a.num_kv_heads;
     const int D = a.head_dim;
+    // block shape: see launch_one
+    const int shape = a.max_rows_per_item > kPrefixTileRows ? 2 : ((a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) ? 1 : 0);
+    const int tile_keys = shape == 1 ? prefix_tile_keys<true>() : prefix_tile_keys<false>();
     CUtensorMap mq, mk, mv;
     {   // Q as (d, g, kv head, sample): a box of (64, G, 1, 128/G) lands as 128 rows ordered sample-major, g fastest
         const cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(G), cuuint64_t(a.num_kv_heads), cuuint64_t(a.num_samples)};
@@ -692,17 +703,17 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
         const cuuint32_t box[4] = {64, cuuint32_t(G), 1, cuuint32_t(kPrefixTileRows / G)};
         if (!encode(fn, &mq, a.q, 4, dims, strides, box, err)) return int(cudaErrorInvalidValue);
     }
-    {   // K and V as (d, kv head, token): a box of (64, 1, 128) is one half of a 128-key tile
+    {   // K and V as (d, kv head, token): a box of (64, 1, tile_keys) is one 64-wide half of a key tile
         const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(a.num_kv_heads), cuuint64_t(a.total_tokens)};
         const cuuint64_t strides[2] = {cuuint64_t(a.stride_head) * 2, cuuint64_t(a.stride_tok) * 2};
-        const cuuint32_t box[3] = {64, 1, cuuint32_t(kPrefixTileKeys)};
+        const cuuint32_t box[3] = {64, 1, cuuint32_t(tile_keys)};
         if (!encode(fn, &mk, a.k, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
         if (!encode(fn, &mv, a.v, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc;
-    if (a.max_rows_per_item > kPrefixTileRows) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
-    else if (a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
+    if (shape == 2) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
+    else if (shape == 1) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
     else rc = D == 128 ? launch_one<128, 0>(a, mq, mk, mv, st) : launch_one<64, 0>(a, mq, mk, mv, st);
     if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));
     return rc;
