@@ -285,3 +285,28 @@ def test_misuse_returns_status_codes_not_faults():
     decode(*good)                                      # and the context is still healthy
     torch.cuda.synchronize()
     plan.check_status()
+
+
+# ------------------------------------------------------------------ seeded random shapes
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_shapes_against_oracle(seed):
+    """Random prompts / samples / lengths / head geometry, every element against the oracle.  The shapes cover
+    all three prefix block shapes (<= 64 rows with long items, <= 128 rows, > 128 rows) and ragged everything."""
+    rng = np.random.default_rng(1000 + seed)
+    D = int(rng.choice([64, 128]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.choice([1, 2, 3]))
+    P = int(rng.integers(1, 5))
+    style = seed % 3
+    if style == 0:      # few samples, long prompts
+        n_samples = rng.integers(0, max(2, 64 // G), size=P); prefix_lens = rng.integers(0, 3000, size=P)
+    elif style == 1:    # around one row tile
+        n_samples = rng.integers(1, max(2, 160 // G), size=P); prefix_lens = rng.integers(0, 700, size=P)
+    else:               # several row tiles (R >= 512 for some prompt)
+        n_samples = rng.integers(1, 40, size=P); n_samples[0] = 520 // G + int(rng.integers(0, 9))
+        prefix_lens = rng.integers(1, 500, size=P)
+    B = int(n_samples.sum())
+    suffix_lens = rng.integers(0, int(rng.choice([40, 300, 1100])), size=B)
+    c = wl.PsaConfig("fuzz", P, 1, G * Hkv, Hkv, D, (1, 1), (0, 1), permute_pages=bool(seed % 2), seed=seed)
+    w = wl.make_workload(c, poison=True, lengths=(prefix_lens, n_samples, suffix_lens))
+    check(w, "f32" if seed % 2 else "bf16", what=f"fuzz{seed} D{D} G{G} Hkv{Hkv} N{list(n_samples)} L{list(prefix_lens)}")
