@@ -99,6 +99,21 @@ typedef struct {
 psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes,
                              const int32_t *prefix_lens, const int32_t *n_samples_per_prefix,
                              const int32_t *suffix_lens, psa_plan_t **out_plan);
+/*
+ * Plan for a CASCADE of shared prefixes: the prompts of the paper's sampling step are themselves layered --
+ * base prompt + demonstrations d_j shared by every task, then the task text shared by that task's N samples
+ * (Algorithm 1, the sampling step; the prompt composer appends the task-specific input last) -- so the big
+ * level can be batched over ALL samples.  A "group" is a run of consecutive tokens of the packed prefix arrays
+ * attended by a run of consecutive samples:
+ *   group g = tokens [T_g, T_g + group_token_len[g]) with T_g = sum of the earlier groups' lengths,
+ *             samples [group_first_sample[g], group_first_sample[g] + group_n_samples[g]).
+ * A sample attends to every group that contains it (at most 4) plus its own suffix; the order of keys does
+ * not matter to the result.  psa_plan_create is the special case "group p = prompt p, groups do not overlap".
+ * All arrays are host memory; num_samples = B.  Everything else (psa_decode, workspaces) is unchanged.
+ */
+psa_status_t psa_plan_create_cascade(const psa_config_t *cfg, int32_t num_groups, const int32_t *group_first_sample,
+                                     const int32_t *group_n_samples, const int32_t *group_token_len, int32_t num_samples,
+                                     const int32_t *suffix_lens, psa_plan_t **out_plan);
 psa_status_t psa_plan_destroy(psa_plan_t *plan);
 psa_status_t psa_plan_get_info(const psa_plan_t *plan, psa_plan_info_t *info);
 

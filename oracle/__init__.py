@@ -37,6 +37,8 @@ class _Problem(ctypes.Structure):
         ("num_prefixes", ctypes.c_int),
         ("prefix_lens", ctypes.c_void_p),
         ("n_samples", ctypes.c_void_p),
+        ("first_sample", ctypes.c_void_p),
+        ("num_samples", ctypes.c_int32),
         ("num_q_heads", ctypes.c_int),
         ("num_kv_heads", ctypes.c_int),
         ("head_dim", ctypes.c_int),
@@ -92,6 +94,12 @@ def _problem(w: dict):
         a = w[name]
         assert a.dtype == np.uint16, f"{name} must hold bf16 bit patterns (uint16)"
         keep[name] = np.ascontiguousarray(a)
+    # prefix groups: explicit (cascade: first_sample given) or one group per prompt, samples in order
+    if "group_first_sample" in w:
+        keep["first_sample"] = _c(w["group_first_sample"], np.int32)
+    else:
+        keep["first_sample"] = np.concatenate([[0], np.cumsum(keep["n_samples"])[:-1]]).astype(np.int32) if len(keep["n_samples"]) else np.zeros(0, np.int32)
+    n_total_samples = len(keep["suffix_lens"])
     Hq, Hkv, D = int(w["num_q_heads"]), int(w["num_kv_heads"]), int(w["head_dim"])
     page = int(w["page_size"])
     # default layouts: prefix [sum L, Hkv, D]; pool [pages, Hkv, page, D]
@@ -99,6 +107,7 @@ def _problem(w: dict):
     qst = w.get("pool_strides", (Hkv * page * D, page * D, D))
     pb = _Problem(
         len(keep["prefix_lens"]), keep["prefix_lens"].ctypes.data, keep["n_samples"].ctypes.data,
+        keep["first_sample"].ctypes.data, n_total_samples,
         Hq, Hkv, D, page, float(w["sm_scale"]),
         keep["q"].ctypes.data, keep["prefix_k"].ctypes.data, keep["prefix_v"].ctypes.data,
         int(pst[0]), int(pst[1]),
@@ -115,7 +124,7 @@ def attend(w: dict, rows=None, n_threads: int = 0):
     """
     lib = _load()
     pb, keep = _problem(w)
-    B = int(np.sum(keep["n_samples"]))
+    B = len(keep["suffix_lens"])
     if rows is None:
         n_rows, rows_ptr = B * pb.num_q_heads, None
     else:
@@ -135,7 +144,7 @@ def weights(w: dict, s: int, h: int):
     """Softmax weights of row (s, h) over its prefix-then-suffix context, fp64."""
     lib = _load()
     pb, keep = _problem(w)
-    cap = int(np.max(keep["prefix_lens"], initial=0)) + int(np.max(keep["suffix_lens"], initial=0)) + 1
+    cap = int(np.sum(keep["prefix_lens"])) + int(np.max(keep["suffix_lens"], initial=0)) + 1
     buf = np.zeros((cap,), dtype=np.float64)
     n = lib.psa_oracle_weights(ctypes.byref(pb), int(s), int(h), buf.ctypes.data, cap)
     if n < 0:

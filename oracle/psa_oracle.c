@@ -21,6 +21,12 @@
  *   lse   = m + ln Z                       (natural logarithm)
  *   empty context: out = 0, lse = -inf
  *
+ * Cascades: the shared part of a context may itself be layered (demonstrations shared by every task, task
+ * text shared by the task's samples: Algorithm 1's sampling step).  A prefix GROUP g is a run of prefix_lens[g]
+ * consecutive tokens of the packed prefix arrays attended by samples [first_sample[g], first_sample[g] +
+ * n_samples[g]); a sample's context is every group that contains it, in group order, then its own tokens.
+ * The flat case (first_sample == NULL) is "group p = prompt p, samples handed out in order".
+ *
  * q, k and v arrive as bf16 bit patterns and are widened exactly.
  * Suffix token t of sample s lives in physical page
  * page_indices[page_indptr[s] + t / page_size], slot t % page_size.
@@ -48,6 +54,8 @@ typedef struct {
     int num_prefixes;
     const int32_t *prefix_lens;   /* [P] */
     const int32_t *n_samples;     /* [P] */
+    const int32_t *first_sample;  /* [P] or NULL (groups are consecutive prompts) */
+    int32_t num_samples;          /* B */
     int num_q_heads, num_kv_heads, head_dim, page_size;
     double sm_scale;
     const uint16_t *q;            /* [B, Hq, D] */
@@ -60,18 +68,52 @@ typedef struct {
     const int32_t *suffix_lens;   /* [B] */
 } psa_oracle_problem;
 
+/* Samples [*first, *first + n_samples[g]) of group g. */
+static int64_t group_first(const psa_oracle_problem *pb, int g)
+{
+    if (pb->first_sample) return pb->first_sample[g];
+    int64_t first = 0;
+    for (int p = 0; p < g; ++p) first += pb->n_samples[p];
+    return first;
+}
+
+/* Address of key / value number j of the context of sample s, kv head `kv`; *n receives the context length
+ * when j < 0.  Walks the groups and then the page table: deliberately the slow, obvious way. */
+static const uint16_t *context_row(const psa_oracle_problem *pb, int s, int kv, int64_t j, int want_v, int64_t *n)
+{
+    int64_t seen = 0, tok_off = 0;
+    for (int g = 0; g < pb->num_prefixes; ++g) {
+        const int64_t first = group_first(pb, g), L = pb->prefix_lens[g];
+        if (s >= first && s < first + pb->n_samples[g]) {
+            if (j >= 0 && j < seen + L) {
+                const uint16_t *base = want_v ? pb->prefix_v : pb->prefix_k;
+                return base + (tok_off + (j - seen)) * pb->prefix_stride_tok + kv * pb->prefix_stride_head;
+            }
+            seen += L;
+        }
+        tok_off += L;
+    }
+    const int64_t S = pb->suffix_lens[s];
+    if (j >= 0 && j < seen + S) {
+        const int64_t t = j - seen;
+        const int64_t page = pb->page_indices[pb->page_indptr[s] + t / pb->page_size];
+        const uint16_t *base = want_v ? pb->pool_v : pb->pool_k;
+        return base + page * pb->pool_stride_page + kv * pb->pool_stride_head + (t % pb->page_size) * pb->pool_stride_tok;
+    }
+    if (n) *n = seen + S;
+    return NULL;
+}
+
 /* One (sample, query head) row, two passes over the concatenated context.
  * weights (optional, length n) receives w_j / Z. Returns the context length. */
-static int64_t attend_row(const psa_oracle_problem *pb, int prompt, int64_t prompt_tok_off,
-                          int s, int h, double *x /* scratch, >= n */,
+static int64_t attend_row(const psa_oracle_problem *pb, int s, int h, double *x /* scratch, >= n */,
                           double *out, double *lse, double *weights)
 {
     const int D = pb->head_dim;
     const int G = pb->num_q_heads / pb->num_kv_heads;
     const int kv = h / G;
-    const int64_t L = pb->prefix_lens[prompt];
-    const int64_t S = pb->suffix_lens[s];
-    const int64_t n = L + S;
+    int64_t n = 0;
+    context_row(pb, s, kv, -1, 0, &n);
     const uint16_t *qrow = pb->q + ((int64_t)s * pb->num_q_heads + h) * D;
 
     for (int d = 0; d < D; ++d) out[d] = 0.0;
@@ -80,15 +122,7 @@ static int64_t attend_row(const psa_oracle_problem *pb, int prompt, int64_t prom
     /* pass 1: logits and their maximum */
     double m = -INFINITY;
     for (int64_t j = 0; j < n; ++j) {
-        const uint16_t *krow;
-        if (j < L) {
-            krow = pb->prefix_k + (prompt_tok_off + j) * pb->prefix_stride_tok + kv * pb->prefix_stride_head;
-        } else {
-            int64_t t = j - L;
-            int64_t page = pb->page_indices[pb->page_indptr[s] + t / pb->page_size];
-            krow = pb->pool_k + page * pb->pool_stride_page + kv * pb->pool_stride_head
-                 + (t % pb->page_size) * pb->pool_stride_tok;
-        }
+        const uint16_t *krow = context_row(pb, s, kv, j, 0, NULL);
         double dot = 0.0;
         for (int d = 0; d < D; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
         x[j] = pb->sm_scale * dot;
@@ -97,15 +131,7 @@ static int64_t attend_row(const psa_oracle_problem *pb, int prompt, int64_t prom
     /* pass 2: weights, normaliser, weighted sum of values */
     double Z = 0.0;
     for (int64_t j = 0; j < n; ++j) {
-        const uint16_t *vrow;
-        if (j < L) {
-            vrow = pb->prefix_v + (prompt_tok_off + j) * pb->prefix_stride_tok + kv * pb->prefix_stride_head;
-        } else {
-            int64_t t = j - L;
-            int64_t page = pb->page_indices[pb->page_indptr[s] + t / pb->page_size];
-            vrow = pb->pool_v + page * pb->pool_stride_page + kv * pb->pool_stride_head
-                 + (t % pb->page_size) * pb->pool_stride_tok;
-        }
+        const uint16_t *vrow = context_row(pb, s, kv, j, 1, NULL);
         double w = exp(x[j] - m);
         x[j] = w;
         Z += w;
@@ -117,18 +143,6 @@ static int64_t attend_row(const psa_oracle_problem *pb, int prompt, int64_t prom
     return n;
 }
 
-/* Locate the prompt a sample belongs to: samples of prompt 0 first, then prompt 1, ... */
-static void locate_sample(const psa_oracle_problem *pb, int s, int *prompt, int64_t *tok_off)
-{
-    int64_t first = 0, off = 0;
-    for (int p = 0; p < pb->num_prefixes; ++p) {
-        if (s < first + pb->n_samples[p]) { *prompt = p; *tok_off = off; return; }
-        first += pb->n_samples[p];
-        off += pb->prefix_lens[p];
-    }
-    *prompt = -1; *tok_off = 0;
-}
-
 /*
  * Attend for a list of rows.  rows[i] = s * Hq + h selects (sample, query head);
  * rows == NULL means all B*Hq rows in order.  out is [n_rows, D] fp64, lse [n_rows].
@@ -138,13 +152,13 @@ static void locate_sample(const psa_oracle_problem *pb, int s, int *prompt, int6
 int psa_oracle_attend(const psa_oracle_problem *pb, const int64_t *rows, int64_t n_rows,
                       double *out, double *lse, int n_threads, int *threads_used)
 {
-    int64_t B = 0, max_ctx = 1;
-    for (int p = 0; p < pb->num_prefixes; ++p) B += pb->n_samples[p];
-    {
-        int64_t maxL = 0, maxS = 0;
-        for (int p = 0; p < pb->num_prefixes; ++p) if (pb->prefix_lens[p] > maxL) maxL = pb->prefix_lens[p];
+    const int64_t B = pb->num_samples;
+    int64_t max_ctx = 1;
+    {   /* no context is longer than all prefix tokens plus the longest suffix */
+        int64_t sumL = 0, maxS = 0;
+        for (int p = 0; p < pb->num_prefixes; ++p) sumL += pb->prefix_lens[p];
         for (int64_t s = 0; s < B; ++s) if (pb->suffix_lens[s] > maxS) maxS = pb->suffix_lens[s];
-        max_ctx = maxL + maxS + 1;
+        max_ctx = sumL + maxS + 1;
     }
     if (rows == NULL) n_rows = B * pb->num_q_heads;
     int failed = 0, team = 1;
@@ -163,10 +177,7 @@ int psa_oracle_attend(const psa_oracle_problem *pb, const int64_t *rows, int64_t
             int64_t r = rows ? rows[i] : i;
             if (!x || r < 0 || r >= B * pb->num_q_heads) { failed = 1; continue; }
             int s = (int)(r / pb->num_q_heads), h = (int)(r % pb->num_q_heads);
-            int prompt; int64_t tok_off;
-            locate_sample(pb, s, &prompt, &tok_off);
-            if (prompt < 0) { failed = 1; continue; }
-            attend_row(pb, prompt, tok_off, s, h, x, out + i * pb->head_dim, lse + i, NULL);
+            attend_row(pb, s, h, x, out + i * pb->head_dim, lse + i, NULL);
         }
         free(x);
     }
@@ -174,19 +185,18 @@ int psa_oracle_attend(const psa_oracle_problem *pb, const int64_t *rows, int64_t
     return failed ? -1 : 0;
 }
 
-/* Softmax weights w_j / Z of one row over its concatenated context (length L_p + S_s). */
+/* Softmax weights w_j / Z of one row over its concatenated context. */
 int64_t psa_oracle_weights(const psa_oracle_problem *pb, int s, int h, double *weights, int64_t capacity)
 {
-    int prompt; int64_t tok_off;
-    locate_sample(pb, s, &prompt, &tok_off);
-    if (prompt < 0) return -1;
-    int64_t n = (int64_t)pb->prefix_lens[prompt] + pb->suffix_lens[s];
+    if (s < 0 || s >= pb->num_samples) return -1;
+    int64_t n = 0;
+    context_row(pb, s, 0, -1, 0, &n);
     if (n > capacity) return -1;
     double *x = (double *)malloc(sizeof(double) * (size_t)(n + 1));
     double *o = (double *)malloc(sizeof(double) * (size_t)pb->head_dim);
     double l;
     if (!x || !o) { free(x); free(o); return -1; }
-    attend_row(pb, prompt, tok_off, s, h, x, o, &l, weights);
+    attend_row(pb, s, h, x, o, &l, weights);
     free(x); free(o);
     return n;
 }

@@ -29,15 +29,19 @@ def gather_context(w: dict, s: int, h: int):
     kv = h // G
     n_samples = np.asarray(w["n_samples"])
     prefix_lens = np.asarray(w["prefix_lens"])
-    first = np.concatenate([[0], np.cumsum(n_samples)])
-    p = int(np.searchsorted(first, s, side="right") - 1)
-    tok_off = int(np.sum(prefix_lens[:p]))
-    L, S = int(prefix_lens[p]), int(w["suffix_lens"][s])
+    # prefix groups: explicit first samples (cascade) or consecutive prompts
+    first = np.asarray(w["group_first_sample"]) if "group_first_sample" in w else np.concatenate([[0], np.cumsum(n_samples)[:-1]])
+    tok = np.concatenate([[0], np.cumsum(prefix_lens)])
+    S = int(w["suffix_lens"][s])
     q = bf16_bits_to_f64(np.asarray(w["q"]).reshape(-1, Hq, D)[s, h])
     pk = np.asarray(w["prefix_k"]).reshape(-1, Hkv, D)
     pv = np.asarray(w["prefix_v"]).reshape(-1, Hkv, D)
-    K = [pk[tok_off + t, kv] for t in range(L)]
-    V = [pv[tok_off + t, kv] for t in range(L)]
+    K, V = [], []
+    for g in range(len(prefix_lens)):
+        if int(first[g]) <= s < int(first[g]) + int(n_samples[g]):
+            K += [pk[t, kv] for t in range(int(tok[g]), int(tok[g + 1]))]
+            V += [pv[t, kv] for t in range(int(tok[g]), int(tok[g + 1]))]
+    L = len(K)
     poolk = np.asarray(w["pool_k"]).reshape(-1, Hkv, page, D)
     poolv = np.asarray(w["pool_v"]).reshape(-1, Hkv, page, D)
     for t in range(S):

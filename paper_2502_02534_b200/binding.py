@@ -15,7 +15,7 @@ PSA_OUT_BF16, PSA_OUT_F32 = 0, 1
 
 # every symbol include/psa.h declares
 EXPORTED_SYMBOLS = [
-    "psa_plan_create", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
+    "psa_plan_create", "psa_plan_create_cascade", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
     "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status",
@@ -68,6 +68,8 @@ def library():
         P = c_void_p
         lib.psa_plan_create.restype = c_int32
         lib.psa_plan_create.argtypes = [POINTER(_Config), c_int32, P, P, P, POINTER(c_void_p)]
+        lib.psa_plan_create_cascade.restype = c_int32
+        lib.psa_plan_create_cascade.argtypes = [POINTER(_Config), c_int32, P, P, P, c_int32, P, POINTER(c_void_p)]
         lib.psa_plan_destroy.restype = c_int32
         lib.psa_plan_destroy.argtypes = [P]
         lib.psa_plan_get_info.restype = c_int32
@@ -140,7 +142,9 @@ class Plan:
 
     def __init__(self, prefix_lens, n_samples_per_prefix, suffix_lens, *, num_q_heads, num_kv_heads, head_dim,
                  page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0, suffix_chunk_tokens=0, prefix_tiles_per_item=0,
-                 prefix_rows_per_item=0):
+                 prefix_rows_per_item=0, groups=None):
+        """``groups`` = (first_sample[], n_samples[], token_len[]) plans a cascade of shared prefixes
+        (psa_plan_create_cascade); ``prefix_lens`` / ``n_samples_per_prefix`` are then ignored."""
         lib = library()
         self.prefix_lens, self.n_samples, self.suffix_len_bounds = _i32(prefix_lens), _i32(n_samples_per_prefix), _i32(suffix_lens)
         self.num_q_heads, self.num_kv_heads, self.head_dim, self.page_size = num_q_heads, num_kv_heads, head_dim, page_size
@@ -150,8 +154,14 @@ class Plan:
                       suffix_chunk_tokens, prefix_tiles_per_item, prefix_rows_per_item, 0)
         handle = c_void_p()
         self._h = None
-        _check(lib.psa_plan_create(ctypes.byref(cfg), len(self.prefix_lens), _ptr(self.prefix_lens), _ptr(self.n_samples),
-                                   _ptr(self.suffix_len_bounds), ctypes.byref(handle)))
+        if groups is None:
+            _check(lib.psa_plan_create(ctypes.byref(cfg), len(self.prefix_lens), _ptr(self.prefix_lens), _ptr(self.n_samples),
+                                       _ptr(self.suffix_len_bounds), ctypes.byref(handle)))
+        else:
+            self.groups = tuple(_i32(a) for a in groups)
+            _check(lib.psa_plan_create_cascade(ctypes.byref(cfg), len(self.groups[0]), _ptr(self.groups[0]), _ptr(self.groups[1]),
+                                               _ptr(self.groups[2]), len(self.suffix_len_bounds), _ptr(self.suffix_len_bounds),
+                                               ctypes.byref(handle)))
         self._h = handle
         self.workspace = None
 

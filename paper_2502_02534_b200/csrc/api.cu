@@ -4,6 +4,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "psa_internal.h"
 
@@ -54,8 +55,9 @@ psa_status_t set_last_error(psa_status_t status, const std::string &message) { r
 
 extern "C" {
 
-psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes, const int32_t *prefix_lens,
-                             const int32_t *n_samples_per_prefix, const int32_t *suffix_lens, psa_plan_t **out_plan)
+static psa_status_t create_impl(const psa_config_t *cfg, int32_t num_groups, const int32_t *first_sample,
+                                const int32_t *n_samples, const int32_t *token_len, int32_t num_samples,
+                                const int32_t *suffix_lens, psa_plan_t **out_plan)
 {
     if (!cfg || !out_plan) return fail(PSA_ERR_INVALID_ARG, "null cfg or out_plan");
     *out_plan = nullptr;
@@ -70,13 +72,36 @@ psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes, cons
     psa_plan *plan = new (std::nothrow) psa_plan();
     if (!plan) return fail(PSA_ERR_INVALID_ARG, "out of host memory");
     std::string err;
-    psa_status_t st = psa::build_plan(c, num_prefixes, prefix_lens, n_samples_per_prefix, suffix_lens, plan, &err);
+    psa_status_t st = psa::build_plan(c, num_groups, first_sample, n_samples, token_len, num_samples, suffix_lens, plan, &err);
     if (st != PSA_OK) {
         delete plan;
         return fail(st, err);
     }
     *out_plan = plan;
     return PSA_OK;
+}
+
+psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes, const int32_t *prefix_lens,
+                             const int32_t *n_samples_per_prefix, const int32_t *suffix_lens, psa_plan_t **out_plan)
+{
+    if (num_prefixes < 0 || (num_prefixes > 0 && !n_samples_per_prefix)) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
+    // prompt p is the prefix group of the next n_samples_per_prefix[p] samples
+    std::vector<int32_t> first(static_cast<size_t>(num_prefixes), 0);
+    int64_t B = 0;
+    for (int32_t p = 0; p < num_prefixes; ++p) {
+        if (n_samples_per_prefix[p] < 0) return fail(PSA_ERR_INVALID_ARG, "negative length or sample count");
+        first[size_t(p)] = int32_t(B);
+        B += n_samples_per_prefix[p];
+        if (B > (1 << 24)) return fail(PSA_ERR_UNSUPPORTED, "problem too large");
+    }
+    return create_impl(cfg, num_prefixes, first.data(), n_samples_per_prefix, prefix_lens, int32_t(B), suffix_lens, out_plan);
+}
+
+psa_status_t psa_plan_create_cascade(const psa_config_t *cfg, int32_t num_groups, const int32_t *group_first_sample,
+                                     const int32_t *group_n_samples, const int32_t *group_token_len, int32_t num_samples,
+                                     const int32_t *suffix_lens, psa_plan_t **out_plan)
+{
+    return create_impl(cfg, num_groups, group_first_sample, group_n_samples, group_token_len, num_samples, suffix_lens, out_plan);
 }
 
 psa_status_t psa_plan_destroy(psa_plan_t *plan)

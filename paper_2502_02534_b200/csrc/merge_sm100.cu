@@ -34,19 +34,34 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
     const int s = row / num_q_heads, h = row % num_q_heads;
     const int kv = h / group, g = h % group;
 
+    // head of the sample's record, then one int4 per prefix level (a sample of a cascade belongs to several groups)
     const int4 *ip = reinterpret_cast<const int4 *>(sample_info + s);
-    const int4 a = __ldg(ip), b = __ldg(ip + 1);
-    const int pre_row0 = a.x, pre_split_stride = a.y, pre_splits = a.z, pre_head_stride = a.w;
-    const int suf_row0 = b.x, suf_chunks = b.y, suf_bound = b.z;
+    const int4 head = __ldg(ip);
+    const int suf_row0 = head.x, suf_chunks = head.y, suf_bound = head.z, n_levels = head.w;
+    int lv_first[kMaxPrefixLevels], lv_stride[kMaxPrefixLevels], lv_end[kMaxPrefixLevels];   // lv_end: running count of splits
+    int n_pre = 0;
+#pragma unroll
+    for (int l = 0; l < kMaxPrefixLevels; ++l) {
+        int4 lv = make_int4(0, 0, 0, 0);
+        if (l < n_levels) lv = __ldg(ip + 1 + l);
+        lv_first[l] = lv.x + kv * lv.w + g;
+        lv_stride[l] = lv.y;
+        n_pre += lv.z;
+        lv_end[l] = n_pre;
+    }
     int S = __ldg(suffix_lens + s);
     S = min(max(S, 0), suf_bound);
     const int n_suf = (S + chunk_tokens - 1) / chunk_tokens;
-    const int n_total = pre_splits + n_suf;
+    const int n_total = n_pre + n_suf;
 
-    const int pre_first = pre_row0 + kv * pre_head_stride + g;
     const int suf_first = suf_row0 + kv * suf_chunks * group + g;
     auto partial_row = [&](int i) {
-        return i < pre_splits ? pre_first + i * pre_split_stride : suf_first + (i - pre_splits) * group;
+        if (i >= n_pre) return suf_first + (i - n_pre) * group;
+        int r = lv_first[0] + i * lv_stride[0];
+#pragma unroll
+        for (int l = 1; l < kMaxPrefixLevels; ++l)
+            if (i >= lv_end[l - 1]) r = lv_first[l] + (i - lv_end[l - 1]) * lv_stride[l];
+        return r;
     };
 
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed

@@ -18,28 +18,32 @@ namespace {
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Prefix: every (prompt, kv head, row group) streams ceil(L_p / 128) key tiles.  With at
-// most T tiles per item the stage takes ceil(items / SMs) waves of (T + overhead) tile
-// steps; pick the T with the smallest estimate, preferring larger T on ties (fewer
-// partial results to write and merge).
-int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::vector<int64_t> &groups, int num_sms)
+// Prefix: every (group, kv head, row group) streams ceil(L / 128) key tiles; with at most T tiles per item a
+// group of `tiles` tiles is cut into ceil(tiles / T) items.  Items are dispatched longest first to the SMs, so
+// the stage takes about max(longest item, sum of items / SMs); every split also costs a partial result per row
+// (4*D bytes written, read again by the merge stage).  Costs are in tile steps of a one-row-tile block (~1.5 us);
+// a step of a two-row-tile block counts 1.6.  Pick the T with the smallest estimate, larger T on ties.
+int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::vector<int64_t> &groups,
+                                 const std::vector<int64_t> &partial_rows_per_split, double step_weight, int head_dim, int num_sms)
 {
     int64_t max_tiles = 0;
     for (int64_t t : tiles) max_tiles = std::max(max_tiles, t);
     if (max_tiles == 0) return 1;
-    const double overhead = 2.0;  // prologue + epilogue of one item, in tile steps
+    const double overhead = 2.0;                                   // prologue + epilogue of one item, in tile steps
+    const double steps_per_partial_row = double(head_dim) * 8.0 / 4.0e12 / 1.5e-6;   // bytes / (4 TB/s) / step time
     double best_cost = std::numeric_limits<double>::infinity();
     int best_T = 1;
     for (int64_t T = 1; T <= max_tiles; ++T) {
-        int64_t items = 0, longest = 0;
+        double sum = 0.0, longest = 0.0, partial = 0.0;
         for (size_t p = 0; p < tiles.size(); ++p) {
             if (tiles[p] == 0) continue;
-            int64_t splits = ceil_div(tiles[p], T);
-            items += groups[p] * splits;
-            longest = std::max(longest, ceil_div(tiles[p], splits));
+            const int64_t splits = ceil_div(tiles[p], T);
+            const double len = step_weight * double(ceil_div(tiles[p], splits)) + overhead;
+            sum += double(groups[p] * splits) * len;
+            longest = std::max(longest, len);
+            partial += double(partial_rows_per_split[p] * splits) * steps_per_partial_row;
         }
-        int64_t waves = ceil_div(items, num_sms);
-        double cost = double(waves) * (double(longest) + overhead);
+        const double cost = std::max(longest, 1.1 * sum / num_sms) + partial;
         if (cost <= best_cost) { best_cost = cost; best_T = int(T); }
     }
     return best_T;
@@ -74,8 +78,9 @@ int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sm
 
 }  // namespace
 
-psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefix_lens, const int32_t *n_samples,
-                        const int32_t *suffix_lens, psa_plan *plan, std::string *err)
+psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first_sample, const int32_t *n_samples,
+                        const int32_t *prefix_lens, int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan,
+                        std::string *err)
 {
     auto fail = [&](psa_status_t st, const char *msg) { if (err) *err = msg; return st; };
     if (cfg.num_q_heads <= 0 || cfg.num_kv_heads <= 0 || cfg.num_q_heads % cfg.num_kv_heads != 0)
@@ -95,17 +100,21 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     if (cfg.prefix_rows_per_item != 0 && cfg.prefix_rows_per_item != 128 && cfg.prefix_rows_per_item != 256)
         return fail(PSA_ERR_INVALID_ARG, "prefix_rows_per_item must be 0, 128 or 256");
     if (cfg.num_sms <= 0) return fail(PSA_ERR_INVALID_ARG, "num_sms must be positive here");
-    if (P < 0 || (P > 0 && (!prefix_lens || !n_samples))) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
+    if (P < 0 || (P > 0 && (!prefix_lens || !n_samples || !first_sample))) return fail(PSA_ERR_INVALID_ARG, "null length arrays");
+    if (num_samples < 0) return fail(PSA_ERR_INVALID_ARG, "negative sample count");
 
     plan->cfg = cfg;
     plan->group = G;
     plan->num_prefixes = P;
-    plan->prefix_lens.assign(prefix_lens, prefix_lens + P);
-    plan->n_samples.assign(n_samples, n_samples + P);
-    int64_t B = 0, total_tokens = 0;
+    plan->group_first_sample.assign(first_sample, first_sample + P);
+    plan->group_n_samples.assign(n_samples, n_samples + P);
+    plan->group_token_len.assign(prefix_lens, prefix_lens + P);
+    const int64_t B = num_samples;
+    int64_t total_tokens = 0;
     for (int p = 0; p < P; ++p) {
         if (prefix_lens[p] < 0 || n_samples[p] < 0) return fail(PSA_ERR_INVALID_ARG, "negative length or sample count");
-        B += n_samples[p];
+        if (first_sample[p] < 0 || int64_t(first_sample[p]) + n_samples[p] > B)
+            return fail(PSA_ERR_INVALID_ARG, "a prefix group reaches outside the samples");
         total_tokens += prefix_lens[p];
     }
     if (B > (1 << 24) || total_tokens > (int64_t(1) << 30)) return fail(PSA_ERR_UNSUPPORTED, "problem too large");
@@ -125,30 +134,35 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
     const int rows_per_item = cfg.prefix_rows_per_item > 0 ? cfg.prefix_rows_per_item
                                                            : (max_rows >= 2 * kPrefixRowsPerItem ? kPrefixRowsPerItem : kPrefixTileRows);
     const int samples_per_group = rows_per_item / G;
-    std::vector<int64_t> tiles(P), groups(P);
+    std::vector<int64_t> tiles(P), groups(P), rows_per_split(P);
     for (int p = 0; p < P; ++p) {
         tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;
         groups[p] = int64_t(cfg.num_kv_heads) * ceil_div(n_samples[p], samples_per_group);
+        rows_per_split[p] = int64_t(cfg.num_kv_heads) * n_samples[p] * G;
     }
-    const int T = cfg.prefix_tiles_per_item > 0 ? cfg.prefix_tiles_per_item : choose_prefix_tiles_per_item(tiles, groups, cfg.num_sms);
+    const int T = cfg.prefix_tiles_per_item > 0
+                      ? cfg.prefix_tiles_per_item
+                      : choose_prefix_tiles_per_item(tiles, groups, rows_per_split, rows_per_item > kPrefixTileRows ? 1.6 : 1.0,
+                                                     cfg.head_dim, cfg.num_sms);
     plan->prefix_tiles_per_item = T;
 
     plan->sample_info.assign(size_t(B), SampleInfo{});
     plan->prefix_items.clear();
     int64_t next_row = 0;  // partial rows are handed out prefix first, then suffix
-    int64_t tok_off = 0, samp_off = 0;
+    int64_t tok_off = 0;
     int longest_item_tiles = 0;
     for (int p = 0; p < P; ++p) {
-        const int64_t N = n_samples[p], L = prefix_lens[p], R = N * G;
+        const int64_t N = n_samples[p], L = prefix_lens[p], R = N * G, samp_off = first_sample[p];
         const int64_t splits = tiles[p] > 0 ? ceil_div(tiles[p], T) : 0;
         const int64_t base = next_row;
-        for (int64_t i = 0; i < N; ++i) {
+        for (int64_t i = 0; splits > 0 && i < N; ++i) {
             SampleInfo &si = plan->sample_info[size_t(samp_off + i)];
-            si.pre_row0 = int32_t(base + i * G);
-            si.pre_split_stride = int32_t(R);
-            si.pre_splits = int32_t(splits);
-            si.pre_head_stride = int32_t(R * splits);
-            si.prompt = p;
+            if (si.n_levels >= kMaxPrefixLevels) return fail(PSA_ERR_UNSUPPORTED, "a sample belongs to more than 4 prefix groups");
+            PrefixLevel &lv = si.level[si.n_levels++];
+            lv.row0 = int32_t(base + i * G);
+            lv.split_stride = int32_t(R);
+            lv.splits = int32_t(splits);
+            lv.head_stride = int32_t(R * splits);
         }
         if (splits > 0) {
             // key tiles are dealt out as evenly as possible: the first `extra` splits get one more
@@ -178,7 +192,6 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *prefi
             next_row += int64_t(cfg.num_kv_heads) * splits * R;
         }
         tok_off += L;
-        samp_off += N;
     }
     plan->prefix_tiles_per_item = std::max(1, longest_item_tiles);
     plan->prefix_max_rows_per_item = 0;

@@ -39,20 +39,26 @@ struct SuffixItem {
 };
 static_assert(sizeof(SuffixItem) == 16, "SuffixItem is read as one int4");
 
-// Where the merge stage finds the partial results of one sample.
-// prefix row of (kv head, split j, g): pre_row0 + kv*pre_head_stride + j*pre_split_stride + g
-// suffix row of (kv head, chunk c, g): suf_row0 + (kv*suf_chunks + c)*G + g
+// Where the merge stage finds the partial results of one sample.  A sample belongs to up to kMaxPrefixLevels
+// shared-prefix groups (one per level of a cascade: demonstrations shared by every task, task text shared by the
+// task's samples, ...).
+// prefix row of (level l, kv head, split j, g): level[l].row0 + kv*level[l].head_stride + j*level[l].split_stride + g
+// suffix row of (kv head, chunk c, g):          suf_row0 + (kv*suf_chunks + c)*G + g
+constexpr int kMaxPrefixLevels = 4;
+struct PrefixLevel {
+    int32_t row0;
+    int32_t split_stride;
+    int32_t splits;
+    int32_t head_stride;
+};
 struct SampleInfo {
-    int32_t pre_row0;
-    int32_t pre_split_stride;
-    int32_t pre_splits;
-    int32_t pre_head_stride;
     int32_t suf_row0;
     int32_t suf_chunks;     // chunks at the planned suffix length
     int32_t suf_len_bound;  // planned suffix length
-    int32_t prompt;
+    int32_t n_levels;
+    PrefixLevel level[kMaxPrefixLevels];
 };
-static_assert(sizeof(SampleInfo) == 32, "SampleInfo is read as two int4");
+static_assert(sizeof(SampleInfo) == 80, "SampleInfo is read as five int4");
 
 struct WorkspaceLayout {
     size_t status_off = 0;       // kStatusWords int32
@@ -73,7 +79,7 @@ struct psa_plan {
     int32_t num_samples = 0;
     int32_t group = 1;  // G
     int64_t total_prefix_tokens = 0;
-    std::vector<int32_t> prefix_lens, n_samples, suffix_len_bounds;
+    std::vector<int32_t> group_first_sample, group_n_samples, group_token_len, suffix_len_bounds;
     std::vector<psa::PrefixItem> prefix_items;
     std::vector<psa::SuffixItem> suffix_items;
     std::vector<psa::SampleInfo> sample_info;
@@ -91,8 +97,11 @@ namespace psa {
 psa_status_t set_last_error(psa_status_t status, const std::string &message);
 
 // plan.cpp
-psa_status_t build_plan(const psa_config_t &cfg, int32_t num_prefixes, const int32_t *prefix_lens,
-                        const int32_t *n_samples, const int32_t *suffix_lens, psa_plan *plan, std::string *err);
+// Shared-prefix group g: `token_len[g]` consecutive tokens of the packed prefix arrays (groups back to back, in
+// order) attended by samples [first_sample[g], first_sample[g] + n_samples[g]).
+psa_status_t build_plan(const psa_config_t &cfg, int32_t num_groups, const int32_t *first_sample, const int32_t *n_samples,
+                        const int32_t *token_len, int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan,
+                        std::string *err);
 
 // Launchers (one per .cu file). All enqueue on `stream` and return a CUDA error code (0 = ok).
 struct PrefixArgs {

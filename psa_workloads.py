@@ -153,6 +153,47 @@ def make_workload(cfg: PsaConfig, poison: bool = False, lengths=None) -> dict:
     return w
 
 
+def make_cascade_workload(cfg: PsaConfig, shared_len: int, poison: bool = False, lengths=None) -> dict:
+    """A two-level cascade: ``shared_len`` tokens attended by EVERY sample (the base prompt and demonstrations that
+    all tasks share) followed by the configuration's per-prompt prefixes (the task text shared by a task's samples).
+    Same dict as make_workload, with the prefix arrays holding group 0 (shared) then the per-prompt groups, and
+      prefix_lens [P+1], n_samples [P+1], group_first_sample [P+1]
+    describing the groups (group g: prefix_lens[g] tokens, samples first..first+n)."""
+    w = make_workload(cfg, poison=poison, lengths=lengths)
+    B = len(w["suffix_lens"])
+    Hkv, D = cfg.num_kv_heads, cfg.head_dim
+    first = np.concatenate([[0], np.cumsum(w["n_samples"])[:-1]]).astype(np.int32)
+    w["prefix_k"] = np.concatenate([normal_bf16((shared_len, Hkv, D), cfg.seed, 7), w["prefix_k"]])
+    w["prefix_v"] = np.concatenate([normal_bf16((shared_len, Hkv, D), cfg.seed, 8), w["prefix_v"]])
+    w["prefix_lens"] = np.concatenate([[shared_len], w["prefix_lens"]]).astype(np.int32)
+    w["n_samples"] = np.concatenate([[B], w["n_samples"]]).astype(np.int32)
+    w["group_first_sample"] = np.concatenate([[0], first]).astype(np.int32)
+    return w
+
+
+def flatten_cascade(w: dict) -> dict:
+    """The same problem without sharing: one prefix per SAMPLE that physically holds every token the sample's
+    groups cover, in group order.  Used to check grouped results against ungrouped ones."""
+    B = len(w["suffix_lens"])
+    tok = np.concatenate([[0], np.cumsum(w["prefix_lens"])])
+    ks, vs, lens = [], [], []
+    for s in range(B):
+        n = 0
+        for g in range(len(w["prefix_lens"])):
+            f = int(w["group_first_sample"][g])
+            if f <= s < f + int(w["n_samples"][g]):
+                ks.append(w["prefix_k"][tok[g]:tok[g + 1]]); vs.append(w["prefix_v"][tok[g]:tok[g + 1]])
+                n += int(w["prefix_lens"][g])
+        lens.append(n)
+    flat = {k: v for k, v in w.items() if k != "group_first_sample"}
+    Hkv, D = int(w["num_kv_heads"]), int(w["head_dim"])
+    flat["prefix_k"] = np.concatenate(ks) if ks else np.zeros((0, Hkv, D), np.uint16)
+    flat["prefix_v"] = np.concatenate(vs) if vs else np.zeros((0, Hkv, D), np.uint16)
+    flat["prefix_lens"] = np.asarray(lens, dtype=np.int32)
+    flat["n_samples"] = np.ones(B, dtype=np.int32)
+    return flat
+
+
 def checksum(w: dict) -> int:
     """Order-sensitive 64-bit checksum of the tensors, to tell runs apart in logs."""
     acc = 1469598103934665603

@@ -18,6 +18,8 @@ def to_device(w):
 
 def make_plan(w, out_dtype="bf16", suffix_bounds=None, **kw):
     from paper_2502_02534_b200 import Plan
+    if "group_first_sample" in w:      # a cascade of shared prefixes
+        kw = dict(kw, groups=(w["group_first_sample"], w["n_samples"], w["prefix_lens"]))
     return Plan(w["prefix_lens"], w["n_samples"], w["suffix_lens"] if suffix_bounds is None else suffix_bounds,
                 num_q_heads=w["num_q_heads"], num_kv_heads=w["num_kv_heads"], head_dim=w["head_dim"],
                 page_size=w["page_size"], sm_scale=w["sm_scale"], out_dtype=out_dtype, **kw)
@@ -29,7 +31,7 @@ def run_gpu(w, out_dtype="bf16", plan=None, dev=None, poison_outputs=True):
     from paper_2502_02534_b200 import decode
     dev = dev or to_device(w)
     plan = plan or make_plan(w, out_dtype)
-    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    B, Hq, D = len(w["suffix_lens"]), w["num_q_heads"], w["head_dim"]
     tdt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
     out = torch.full((B, Hq, D), float("nan"), dtype=tdt, device="cuda")
     lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")

@@ -310,3 +310,36 @@ def test_random_shapes_against_oracle(seed):
     c = wl.PsaConfig("fuzz", P, 1, G * Hkv, Hkv, D, (1, 1), (0, 1), permute_pages=bool(seed % 2), seed=seed)
     w = wl.make_workload(c, poison=True, lengths=(prefix_lens, n_samples, suffix_lens))
     check(w, "f32" if seed % 2 else "bf16", what=f"fuzz{seed} D{D} G{G} Hkv{Hkv} N{list(n_samples)} L{list(prefix_lens)}")
+
+
+# ------------------------------------------------------------------ cascades of shared prefixes
+@pytest.mark.parametrize("shared_len,n_prompts,n_samples", [(700, 4, 8), (129, 3, 40), (2000, 16, 4), (64, 2, 150)])
+def test_two_level_cascade_against_oracle(shared_len, n_prompts, n_samples):
+    """Level 0 (demonstrations shared by every task's samples) batched over ALL samples, level 1 per prompt."""
+    c = cfg(num_prefixes=n_prompts, samples_per_prefix=n_samples, prefix_len=(50, 400), suffix_len=(0, 120),
+            num_q_heads=8, num_kv_heads=2, permute_pages=True, seed=21)
+    w = wl.make_cascade_workload(c, shared_len=shared_len, poison=True)
+    eo, el = check(w, "f32", what=f"cascade {shared_len}/{n_prompts}x{n_samples}")
+    # the cascade must agree with the same keys planned without sharing (one prefix per sample)
+    if n_prompts * n_samples <= 64:
+        flat = wl.flatten_cascade(w)
+        out_c, lse_c, _ = run_gpu(w, "f32")
+        out_f, lse_f, _ = run_gpu(flat, "f32")
+        assert np.max(np.abs(out_c - out_f)) <= 2e-3 and np.max(np.abs(lse_c - lse_f)) <= 1e-4
+
+
+def test_cascade_with_overlapping_unnested_groups_and_five_levels_rejected():
+    from paper_2502_02534_b200 import Plan, PsaError
+    c = cfg(num_prefixes=1, samples_per_prefix=6, prefix_len=(10, 10), suffix_len=(0, 30), seed=4)
+    w = wl.make_workload(c, poison=True)
+    lens = np.array([100, 37, 260], np.int32)
+    w["prefix_lens"] = lens; w["n_samples"] = np.array([6, 3, 4], np.int32); w["group_first_sample"] = np.array([0, 1, 2], np.int32)
+    w["prefix_k"] = wl.normal_bf16((int(lens.sum()), 2, 128), 5, 2); w["prefix_v"] = wl.normal_bf16((int(lens.sum()), 2, 128), 5, 3)
+    check(w, "f32", what="overlapping groups")
+    with pytest.raises(PsaError) as e:
+        Plan([], [], [0, 0], num_q_heads=8, num_kv_heads=2, head_dim=128, num_sms=148,
+             groups=([0, 0, 0, 0, 0], [2, 2, 2, 2, 2], [5, 5, 5, 5, 5]))
+    assert e.value.status == 2
+    with pytest.raises(PsaError) as e:
+        Plan([], [], [0, 0], num_q_heads=8, num_kv_heads=2, head_dim=128, num_sms=148, groups=([1], [2], [5]))
+    assert e.value.status == 1

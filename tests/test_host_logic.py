@@ -106,3 +106,24 @@ def test_empty_problems_plan_cleanly():
     assert plan.info.num_prefix_items == 0 and plan.info.num_suffix_items == 0 and plan.info.kernel_launches == 0
     plan = make_plan([0, 5], [3, 0], [0, 0, 0])
     assert plan.info.num_prefix_items == 0 and plan.info.num_suffix_items == 0 and plan.info.kernel_launches == 1
+
+
+def test_cascade_plan_covers_every_group_key_once_and_limits_levels():
+    from paper_2502_02534_b200 import Plan, PsaError
+    first, n, lens = [0, 0, 4, 2], [8, 4, 4, 3], [1000, 130, 77, 300]       # nested and overlapping groups
+    S = [5] * 8
+    plan = Plan([], [], S, num_q_heads=8, num_kv_heads=2, head_dim=128, num_sms=148, groups=(first, n, lens))
+    items = plan.prefix_items()
+    tok = np.concatenate([[0], np.cumsum(lens)])
+    G = 4
+    for g in range(4):
+        cover = np.zeros((2, n[g] * G, lens[g]), dtype=np.int8)
+        for t0, nk, kv, s0, nr, prow, grp, split in items[items[:, 6] == g]:
+            r0 = (s0 - first[g]) * G
+            assert first[g] <= s0 and r0 + nr <= n[g] * G and tok[g] <= t0 and t0 + nk <= tok[g + 1]
+            cover[kv, r0:r0 + nr, t0 - tok[g]:t0 - tok[g] + nk] += 1
+        assert (cover == 1).all()
+    rows = np.concatenate([np.arange(p, p + nr) for _, _, _, _, nr, p, _, _ in items])
+    assert len(set(rows.tolist())) == len(rows)
+    with pytest.raises(PsaError):
+        Plan([], [], S, num_q_heads=8, num_kv_heads=2, head_dim=128, num_sms=148, groups=([0], [9], [10]))

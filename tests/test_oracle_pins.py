@@ -324,3 +324,44 @@ def test_definition_matches_numpy_restatement_on_config1():
         x, V = rec.logits(w, s, h)
         o, m, l = rec.task2_deferred(x, V)
         assert np.allclose(o, out[r], rtol=0, atol=TOL) and abs(m + math.log(l) - lse[r]) < TOL
+
+
+# ---------------------------------------------------------------- cascades of shared prefixes
+def test_cascade_equals_the_same_keys_without_sharing():
+    """Grouped (cascade) contexts against the flat path pinned above: every sample's keys copied out physically."""
+    cfg = tiny_cfg(num_prefixes=3, samples_per_prefix=2, prefix_len=(2, 9), suffix_len=(0, 7), seed=13)
+    w = wl.make_cascade_workload(cfg, shared_len=6, poison=True)
+    assert list(w["n_samples"]) == [6, 2, 2, 2] and list(w["group_first_sample"]) == [0, 0, 2, 4]
+    out, lse, _ = oracle.attend(w)
+    flat = wl.flatten_cascade(w)
+    assert list(flat["prefix_lens"]) == [6 + int(w["prefix_lens"][1 + s // 2]) for s in range(6)]
+    fo, fl, _ = oracle.attend(flat)
+    assert np.allclose(out, fo, rtol=0, atol=TOL) and np.allclose(lse, fl, rtol=0, atol=TOL)
+    for s in range(6):                       # and against the Python streaming form on the grouped layout
+        x, V = rec.logits(w, s, 3)
+        o, m, l = rec.task2_deferred(x, V)
+        assert np.allclose(o, out[s * 4 + 3], rtol=0, atol=TOL) and abs(m + math.log(l) - lse[s * 4 + 3]) < TOL
+        assert len(x) == 6 + int(w["prefix_lens"][1 + s // 2]) + int(w["suffix_lens"][s])
+
+
+def test_cascade_counts_every_token_of_every_level_once():
+    # equal keys => uniform weights; V[..., 0] = token id => out[0] = mean id over the sample's groups and suffix
+    cfg = tiny_cfg(num_prefixes=2, samples_per_prefix=2, prefix_len=(3, 5), suffix_len=(0, 0), seed=2)
+    w = wl.make_cascade_workload(cfg, shared_len=4)
+    w["prefix_k"][:] = bits(0.25)
+    n_tok = w["prefix_k"].shape[0]
+    for t in range(n_tok):
+        w["prefix_v"][t, :, 0] = bits(float(t))
+    out, lse, _ = oracle.attend(w)
+    tok = np.concatenate([[0], np.cumsum(w["prefix_lens"])])
+    for s in range(4):
+        ids = list(range(0, 4)) + list(range(int(tok[1 + s // 2]), int(tok[2 + s // 2])))
+        assert np.allclose(out.reshape(4, 4, -1)[s, :, 0], np.mean(ids), rtol=0, atol=1e-11)
+    # overlapping groups that are not nested also work: samples 1..2 get an extra group
+    w2 = dict(w)
+    lens = np.array(list(w["prefix_lens"]), np.int32)
+    w2["prefix_lens"] = lens; w2["n_samples"] = np.array([4, 2, 2], np.int32); w2["group_first_sample"] = np.array([0, 1, 2], np.int32)
+    out2, _, _ = oracle.attend(w2)
+    want = {0: [0, 1, 2, 3], 1: list(range(0, 4 + int(lens[1]))), 2: list(range(0, int(tok[3]))), 3: [0, 1, 2, 3] + list(range(int(tok[2]), int(tok[3])))}
+    for s in range(4):
+        assert np.allclose(out2.reshape(4, 4, -1)[s, :, 0], np.mean(want[s]), rtol=0, atol=1e-11)
