@@ -232,6 +232,14 @@ psa_status_t psa_decode_host(const psa_plan_t *plan, const void *q_host,
  */
 psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cuda_stream);
 
+/*
+ * Self-test of the device-side error path (no counterpart in the paper).  Enqueues one tiny kernel whose only
+ * wait is on a barrier that nothing completes; the wait gives up after `limit_ns` (<= 1 s), the kernel writes
+ * PSA_ERR_TIMEOUT into the status word of `workspace` and exits normally.  psa_check_status then reports and
+ * clears it, and the context stays usable.  This is how the bounded waits of the prefix stage fail, too.
+ */
+psa_status_t psa_selftest_bounded_wait(void *workspace, size_t workspace_bytes, uint64_t limit_ns, void *cuda_stream);
+
 const char *psa_status_string(psa_status_t status);
 const char *psa_last_error_message(void); /* thread-local detail of the last non-OK return */
 int32_t psa_version(void);

@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -98,6 +98,8 @@ def library():
         lib.psa_decode_host.argtypes = [P, P, P, P, c_int64, P, P, c_int64, P, P, c_int64, P, P, P, P, c_size_t, P, c_size_t, P]
         lib.psa_check_status.restype = c_int32
         lib.psa_check_status.argtypes = [P, P, P]
+        lib.psa_selftest_bounded_wait.restype = c_int32
+        lib.psa_selftest_bounded_wait.argtypes = [P, c_size_t, ctypes.c_uint64, P]
         lib.psa_status_string.restype = c_char_p
         lib.psa_status_string.argtypes = [c_int32]
         lib.psa_last_error_message.restype = c_char_p
@@ -204,6 +206,10 @@ class Plan:
         _check(library().psa_plan_bind_workspace(self._h, _ptr(workspace), workspace.numel(), _stream_ptr(stream)))
         self.workspace = workspace
         return workspace
+
+    def selftest_bounded_wait(self, limit_ns=2_000_000, stream=None):
+        """Enqueue the kernel whose wait can never be satisfied; check_status() must then raise PSA_ERR_TIMEOUT."""
+        _check(library().psa_selftest_bounded_wait(_ptr(self.workspace), self.workspace.numel(), int(limit_ns), _stream_ptr(stream)))
 
     def check_status(self, stream=None):
         _check(library().psa_check_status(self._h, _ptr(self.workspace), _stream_ptr(stream)))

@@ -358,6 +358,16 @@ psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cud
     return PSA_OK;
 }
 
+psa_status_t psa_selftest_bounded_wait(void *workspace, size_t workspace_bytes, uint64_t limit_ns, void *cuda_stream)
+{
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < sizeof(int32_t) * psa::kStatusWords)
+        return fail(PSA_ERR_WORKSPACE, "workspace must be a 256-byte aligned device buffer of at least 256 bytes");
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return fail(PSA_ERR_INVALID_ARG, "limit_ns must be in (0, 1e9]");
+    const int rc = psa::launch_bounded_wait_selftest(static_cast<int32_t *>(workspace), limit_ns, cuda_stream);
+    if (rc != 0) return cuda_fail(cudaError_t(rc), "self-test launch");
+    return PSA_OK;
+}
+
 const char *psa_status_string(psa_status_t status)
 {
     switch (status) {

@@ -69,7 +69,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false when the limit passed or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
@@ -77,7 +78,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            if (global_timer_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -614,6 +615,23 @@ prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_c
     prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
 }
 
+// Self-test of the bounded wait: one block waits on a barrier that nothing ever arrives on.  The wait must give
+// up after `limit_ns`, report PSA_ERR_TIMEOUT through the status word and let the block exit normally.
+__global__ void bounded_wait_selftest_kernel(int *status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag)) atomicCAS(status, 0, int(PSA_ERR_TIMEOUT));
+}
+
 // ---------------------------------------------------------------- host side
 using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -685,6 +703,12 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
 }
 
 }  // namespace
+
+int launch_bounded_wait_selftest(int32_t *status, unsigned long long limit_ns, void *stream)
+{
+    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(status, limit_ns);
+    return int(cudaGetLastError());
+}
 
 int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
 {

@@ -117,6 +117,7 @@ struct PrefixArgs {
     int32_t *status;                 // device
 };
 int launch_prefix(const PrefixArgs &a, void *stream, std::string *err);
+int launch_bounded_wait_selftest(int32_t *status, unsigned long long limit_ns, void *stream);
 
 struct SuffixArgs {
     const void *q, *pool_k, *pool_v;

@@ -343,3 +343,22 @@ def test_cascade_with_overlapping_unnested_groups_and_five_levels_rejected():
     with pytest.raises(PsaError) as e:
         Plan([], [], [0, 0], num_q_heads=8, num_kv_heads=2, head_dim=128, num_sms=148, groups=([1], [2], [5]))
     assert e.value.status == 1
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing satisfies gives up after its limit, raises PSA_ERR_TIMEOUT through the status word,
+    and the next decode on the same context and workspace is correct."""
+    import time
+    from paper_2502_02534_b200 import PsaError
+    w = wl.make_workload(cfg(), poison=True)
+    dev = to_device(w)
+    plan = make_plan(w, "f32")
+    out, lse, _ = run_gpu(w, "f32", plan=plan, dev=dev)
+    t0 = time.perf_counter()
+    plan.selftest_bounded_wait(limit_ns=2_000_000)           # 2 ms
+    with pytest.raises(PsaError) as e:
+        plan.check_status()
+    assert e.value.status == 5 and time.perf_counter() - t0 < 1.0
+    plan.check_status()                                      # cleared
+    out2, lse2, _ = run_gpu(w, "f32", plan=plan, dev=dev)
+    assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
