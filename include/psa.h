@@ -233,6 +233,20 @@ psa_status_t psa_decode_host(const psa_plan_t *plan, const void *q_host,
 psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cuda_stream);
 
 /*
+ * The step after the path: append one new token per sample to the paged suffix K/V (each of the paper's samples
+ * grows by one token per decode step, up to 1024: appendix "Experiment details").  For every sample s, the rows
+ * new_k[s], new_v[s] ([B, Hkv, D] bf16 device, contiguous) are written to position S_s = suffix_lens[s] of the
+ * sample's page list and suffix_lens[s] becomes S_s + 1 (device memory, in place), all on `cuda_stream`.
+ * The page for position S_s must already be in the sample's page list, and S_s must be below the bound the plan
+ * was made with; otherwise that sample is left untouched and the status word reports PSA_ERR_BOUNDS
+ * (psa_check_status).  The plan itself does not change: psa_decode may follow immediately.
+ */
+psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void *new_v,
+                           void *suffix_k_pool, void *suffix_v_pool, const int64_t pool_strides[3],
+                           const int32_t *page_indptr, const int32_t *page_indices, int32_t *suffix_lens,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Self-test of the device-side error path (no counterpart in the paper).  Enqueues one tiny kernel whose only
  * wait is on a barrier that nothing completes; the wait gives up after `limit_ns` (<= 1 s), the kernel writes
  * PSA_ERR_TIMEOUT into the status word of `workspace` and exits normally.  psa_check_status then reports and

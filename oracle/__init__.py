@@ -150,3 +150,25 @@ def weights(w: dict, s: int, h: int):
     if n < 0:
         raise RuntimeError("psa_oracle_weights failed")
     return buf[:n].copy()
+
+
+def append_kv(w: dict, new_k: np.ndarray, new_v: np.ndarray) -> dict:
+    """The step after the path, as plainly as possible: sample s's new K/V rows ([B, Hkv, D] bf16 bits) go to
+    position S_s of its page list (page S_s // page_size, slot S_s % page_size) and S_s grows by one.
+    Returns a new workload dict with copied pools and lengths; the input is left alone."""
+    page = int(w["page_size"])
+    out = dict(w)
+    out["pool_k"] = np.array(w["pool_k"], copy=True)
+    out["pool_v"] = np.array(w["pool_v"], copy=True)
+    lens = np.array(w["suffix_lens"], dtype=np.int32, copy=True)
+    for s in range(len(lens)):
+        S = int(lens[s])
+        pages = w["page_indices"][int(w["page_indptr"][s]): int(w["page_indptr"][s + 1])]
+        if S // page >= len(pages):
+            raise IndexError(f"sample {s} has no page for position {S}")
+        pg = int(pages[S // page])
+        out["pool_k"][pg, :, S % page, :] = new_k[s]
+        out["pool_v"][pg, :, S % page, :] = new_v[s]
+        lens[s] = S + 1
+    out["suffix_lens"] = lens
+    return out

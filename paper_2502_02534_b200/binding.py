@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -98,6 +98,8 @@ def library():
         lib.psa_decode_host.argtypes = [P, P, P, P, c_int64, P, P, c_int64, P, P, c_int64, P, P, P, P, c_size_t, P, c_size_t, P]
         lib.psa_check_status.restype = c_int32
         lib.psa_check_status.argtypes = [P, P, P]
+        lib.psa_append_kv.restype = c_int32
+        lib.psa_append_kv.argtypes = [P, P, P, P, P, POINTER(c_int64), P, P, P, P, c_size_t, P]
         lib.psa_selftest_bounded_wait.restype = c_int32
         lib.psa_selftest_bounded_wait.argtypes = [P, c_size_t, ctypes.c_uint64, P]
         lib.psa_status_string.restype = c_char_p
@@ -265,6 +267,17 @@ def decode_static(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_poo
     _check(library().psa_decode_static(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, _ptr(suffix_k_pool),
                                        _ptr(suffix_v_pool), qst, _ptr(page_indptr), _ptr(page_indices),
                                        _ptr(suffix_lens), _ptr(out), _ptr(lse), _stream_ptr(stream)))
+
+
+def append_kv(plan: Plan, new_k, new_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens, *,
+              pool_strides=None, stream=None):
+    """psa_append_kv: one new token per sample goes to position suffix_lens[s]; suffix_lens is incremented in place."""
+    if plan.workspace is None:
+        plan.bind_workspace(stream=stream)
+    qst = _strides(pool_strides or default_pool_strides(plan), 3)
+    _check(library().psa_append_kv(plan.handle, _ptr(new_k), _ptr(new_v), _ptr(suffix_k_pool), _ptr(suffix_v_pool), qst,
+                                   _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens), _ptr(plan.workspace),
+                                   plan.workspace.numel(), _stream_ptr(stream)))
 
 
 def decode_host(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,

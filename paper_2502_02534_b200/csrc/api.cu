@@ -358,6 +358,33 @@ psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cud
     return PSA_OK;
 }
 
+psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void *new_v, void *suffix_k_pool,
+                           void *suffix_v_pool, const int64_t pool_strides[3], const int32_t *page_indptr,
+                           const int32_t *page_indices, int32_t *suffix_lens, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream)
+{
+    Carved c;
+    psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
+    if (st != PSA_OK) return st;
+    if (plan->num_samples == 0) return PSA_OK;
+    if (!new_k || !new_v || !suffix_k_pool || !suffix_v_pool || !pool_strides || !page_indptr || !page_indices || !suffix_lens)
+        return fail(PSA_ERR_INVALID_ARG, "null append argument");
+    if (!aligned(new_k, 16) || !aligned(new_v, 16) || !aligned(suffix_k_pool, 16) || !aligned(suffix_v_pool, 16))
+        return fail(PSA_ERR_INVALID_ARG, "new_k, new_v and the pools must be 16-byte aligned");
+    for (int i = 0; i < 3; ++i)
+        if (pool_strides[i] <= 0 || pool_strides[i] % 8) return fail(PSA_ERR_INVALID_ARG, "pool strides must be positive multiples of 8 elements");
+    psa::AppendArgs a{};
+    a.new_k = new_k; a.new_v = new_v; a.pool_k = suffix_k_pool; a.pool_v = suffix_v_pool;
+    a.stride_page = pool_strides[0]; a.stride_head = pool_strides[1]; a.stride_tok = pool_strides[2];
+    a.page_indptr = page_indptr; a.page_indices = page_indices; a.suffix_lens = suffix_lens;
+    a.sample_info = c.sample_info;
+    a.num_samples = plan->num_samples; a.num_kv_heads = plan->cfg.num_kv_heads; a.head_dim = plan->cfg.head_dim;
+    a.status = c.status;
+    const int rc = psa::launch_append(a, cuda_stream);
+    if (rc != 0) return cuda_fail(cudaError_t(rc), "append launch");
+    return PSA_OK;
+}
+
 psa_status_t psa_selftest_bounded_wait(void *workspace, size_t workspace_bytes, uint64_t limit_ns, void *cuda_stream)
 {
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < sizeof(int32_t) * psa::kStatusWords)

@@ -1,0 +1,64 @@
+// Step after the path: append one generated token's K and V per sample to the paged suffix pool.
+//
+// The paper's samples each grow by one token per decode step (appendix "Experiment details": at most 1024
+// output tokens per sample), so between two psa_decode calls every sample's new K/V rows go to position S_s of
+// its page list and S_s becomes S_s + 1.  The plan's suffix lengths are upper bounds, so the same plan serves
+// every step of the loop until a sample reaches its bound.
+//
+// One block per sample: it reads S_s once, copies H_kv x D bf16 for K and for V with 16-byte vectors, and
+// only then stores S_s + 1.  A sample that is already at its planned bound, or whose page list has no page for
+// the new position, is left untouched and PSA_ERR_BOUNDS is raised in the status word.
+#include <cuda_runtime.h>
+
+#include "psa_internal.h"
+
+namespace psa {
+namespace {
+
+__global__ void __launch_bounds__(128)
+append_kernel(const uint4 *__restrict__ new_k, const uint4 *__restrict__ new_v, uint4 *__restrict__ pool_k,
+              uint4 *__restrict__ pool_v, int64_t stride_page, int64_t stride_head, int64_t stride_tok,
+              const int32_t *__restrict__ page_indptr, const int32_t *__restrict__ page_indices,
+              int32_t *__restrict__ suffix_lens, const SampleInfo *__restrict__ sample_info, int num_kv_heads, int head_dim,
+              int *__restrict__ status)
+{
+    const int s = blockIdx.x;
+    __shared__ int sh_pos, sh_page;
+    if (threadIdx.x == 0) {
+        const int S = suffix_lens[s];
+        const int first = page_indptr[s], n_pages = page_indptr[s + 1] - first;
+        const bool ok = S >= 0 && S < sample_info[s].suf_len_bound && S / kPageSize < n_pages;
+        sh_pos = ok ? S : -1;
+        sh_page = ok ? page_indices[first + S / kPageSize] : 0;
+        if (!ok) atomicCAS(status, 0, int(PSA_ERR_BOUNDS));
+    }
+    __syncthreads();
+    const int pos = sh_pos;
+    if (pos < 0) return;
+    const int vec_per_head = head_dim / 8;   // 16-byte vectors per (token, head)
+    // strides are multiples of 8 elements, so element offsets divide into uint4 units exactly
+    const int64_t base = (int64_t(sh_page) * stride_page + int64_t(pos % kPageSize) * stride_tok) / 8;
+    for (int i = threadIdx.x; i < num_kv_heads * vec_per_head; i += blockDim.x) {
+        const int kv = i / vec_per_head, v = i % vec_per_head;
+        const int64_t dst = base + int64_t(kv) * (stride_head / 8) + v;
+        const int64_t src = (int64_t(s) * num_kv_heads + kv) * vec_per_head + v;
+        pool_k[dst] = new_k[src];
+        pool_v[dst] = new_v[src];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) suffix_lens[s] = pos + 1;
+}
+
+}  // namespace
+
+int launch_append(const AppendArgs &a, void *stream)
+{
+    if (a.num_samples == 0) return 0;
+    append_kernel<<<a.num_samples, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4 *>(a.new_k), static_cast<const uint4 *>(a.new_v), static_cast<uint4 *>(a.pool_k),
+        static_cast<uint4 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok, a.page_indptr, a.page_indices,
+        a.suffix_lens, a.sample_info, a.num_kv_heads, a.head_dim, a.status);
+    return int(cudaGetLastError());
+}
+
+}  // namespace psa

@@ -145,4 +145,16 @@ struct MergeArgs {
 };
 int launch_merge(const MergeArgs &a, void *stream, std::string *err);
 
+struct AppendArgs {
+    const void *new_k, *new_v;   // [B, Hkv, D] bf16, device
+    void *pool_k, *pool_v;
+    int64_t stride_page, stride_head, stride_tok;  // elements
+    const int32_t *page_indptr, *page_indices;
+    int32_t *suffix_lens;        // in/out
+    const SampleInfo *sample_info;
+    int32_t num_samples, num_kv_heads, head_dim;
+    int32_t *status;
+};
+int launch_append(const AppendArgs &a, void *stream);
+
 }  // namespace psa

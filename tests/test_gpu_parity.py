@@ -362,3 +362,42 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     plan.check_status()                                      # cleared
     out2, lse2, _ = run_gpu(w, "f32", plan=plan, dev=dev)
     assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_decode_append_decode_loop_reuses_one_plan():
+    """Three decode steps with a token appended to every sample in between, one plan made for the final lengths:
+    pools and lengths bit-exact against the oracle's append, attention within tolerance at every step."""
+    import torch
+    from paper_2502_02534_b200 import PsaError, append_kv
+    steps = 3
+    c = cfg(samples_per_prefix=9, suffix_len=(3, 200), permute_pages=True)
+    w = wl.make_workload(c, poison=False)                      # page lists sized for the bounds
+    bounds = np.array(w["suffix_lens"]).copy()
+    w["suffix_lens"] = (bounds - steps).astype(np.int32)
+    plan = make_plan(w, "f32", suffix_bounds=bounds)
+    dev = to_device(w)
+    B, Hkv, D = 9, w["num_kv_heads"], w["head_dim"]
+    for k in range(steps + 1):
+        out, lse, _ = run_gpu(w, "f32", plan=plan, dev=dev)
+        ref_o, ref_l, _ = oracle.attend(w)
+        assert_close(out, lse, ref_o, ref_l, f"loop step {k}")
+        if k == steps:
+            break
+        new_k = wl.normal_bf16((B, Hkv, D), 70 + k, 1); new_v = wl.normal_bf16((B, Hkv, D), 70 + k, 2)
+        w = oracle.append_kv(w, new_k, new_v)
+        nk = torch.from_numpy(new_k.view(np.int16)).cuda().view(torch.bfloat16)
+        nv = torch.from_numpy(new_v.view(np.int16)).cuda().view(torch.bfloat16)
+        append_kv(plan, nk, nv, dev["pool_k"], dev["pool_v"], dev["page_indptr"], dev["page_indices"], dev["suffix_lens"])
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert np.array_equal(dev["suffix_lens"].cpu().numpy(), w["suffix_lens"])
+        assert np.array_equal(dev["pool_k"].view(torch.int16).cpu().numpy().view(np.uint16), w["pool_k"])
+        assert np.array_equal(dev["pool_v"].view(torch.int16).cpu().numpy().view(np.uint16), w["pool_v"])
+    # every sample is at its bound now: one more append must change nothing and report PSA_ERR_BOUNDS
+    before = dev["pool_k"].clone()
+    append_kv(plan, nk, nv, dev["pool_k"], dev["pool_v"], dev["page_indptr"], dev["page_indices"], dev["suffix_lens"])
+    torch.cuda.synchronize()
+    with pytest.raises(PsaError) as e:
+        plan.check_status()
+    assert e.value.status == 6
+    assert torch.equal(before, dev["pool_k"]) and np.array_equal(dev["suffix_lens"].cpu().numpy(), bounds)

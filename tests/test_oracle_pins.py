@@ -365,3 +365,25 @@ def test_cascade_counts_every_token_of_every_level_once():
     want = {0: [0, 1, 2, 3], 1: list(range(0, 4 + int(lens[1]))), 2: list(range(0, int(tok[3]))), 3: [0, 1, 2, 3] + list(range(int(tok[2]), int(tok[3])))}
     for s in range(4):
         assert np.allclose(out2.reshape(4, 4, -1)[s, :, 0], np.mean(want[s]), rtol=0, atol=1e-11)
+
+
+def test_append_puts_the_new_token_last_in_every_context():
+    cfg = tiny_cfg(samples_per_prefix=4, suffix_len=(1, 9))
+    w = wl.make_workload(cfg)                       # pages exist for lengths up to the drawn ones
+    full = np.array(w["suffix_lens"]).copy()
+    w["suffix_lens"] = np.maximum(full - 1, 0).astype(np.int32)   # one slot short of what the pages hold
+    grow = full > 0
+    new_k = wl.normal_bf16((4, 2, 8), 99, 1); new_v = wl.normal_bf16((4, 2, 8), 99, 2)
+    w2 = oracle.append_kv(w, new_k, new_v) if grow.all() else None
+    if w2 is None:
+        pytest.skip("a sample drew length 0")
+    assert list(w2["suffix_lens"]) == list(w["suffix_lens"] + 1) and w["pool_k"] is not w2["pool_k"]
+    for s in range(4):
+        for h in range(4):
+            q, K, V = rec.gather_context(w2, s, h)
+            q0, K0, V0 = rec.gather_context(w, s, h)
+            assert np.array_equal(K[:-1], K0) and np.array_equal(V[:-1], V0)
+            assert np.array_equal(K[-1], rec.bf16_bits_to_f64(new_k[s, h // 2])) and np.array_equal(V[-1], rec.bf16_bits_to_f64(new_v[s, h // 2]))
+    with pytest.raises(IndexError):
+        w3 = dict(w); w3["suffix_lens"] = (np.array(w["page_indptr"][1:]) - np.array(w["page_indptr"][:-1])) * 4
+        oracle.append_kv(w3, new_k, new_v)
