@@ -50,6 +50,7 @@ psa_status_t carve(const psa_plan_t *plan, void *workspace, size_t bytes, Carved
 }  // namespace
 
 namespace psa {
+int PerDeviceOnce::device_ordinal(int *dev) { return int(cudaGetDevice(dev)); }
 psa_status_t set_last_error(psa_status_t status, const std::string &message) { return fail(status, message); }
 }  // namespace psa
 

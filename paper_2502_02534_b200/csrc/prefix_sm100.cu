@@ -83,7 +83,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
 {
@@ -678,15 +677,14 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     // shape get the smallest block so that a suffix block fits beside it on the SM
     constexpr int ring = prefix_ring<D, kTwo, kShape == 1>();
     static_assert(L::total(ring) <= 227 * 1024 && L::min_ring() <= ring, "shared memory plan does not fit");
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce once;   // per instantiation
+    const int cfg_rc = once.ensure([&] {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total(ring));
-        if (e != cudaSuccess) return int(e);
         // ask for the largest shared-memory carve-out so that a suffix block can share the SM
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return int(e);
-        configured = true;
-    }
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        return int(e);
+    });
+    if (cfg_rc != 0) return cfg_rc;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(a.num_items);

@@ -2,6 +2,7 @@
 // Nothing here is part of the public interface (include/psa.h).
 #pragma once
 
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 #include <string>
@@ -95,6 +96,27 @@ namespace psa {
 
 // api.cu: records the thread-local message psa_last_error_message returns; returns `status`
 psa_status_t set_last_error(psa_status_t status, const std::string &message);
+
+// Kernel attributes (dynamic shared memory size, carve-out preference) are per device: this remembers, for one
+// kernel instantiation, on which devices they have been set.  Thread-safe.
+struct PerDeviceOnce {
+    static constexpr int kMaxDevices = 64;
+    std::atomic<unsigned char> done[kMaxDevices];
+    PerDeviceOnce() { for (auto &d : done) d.store(0); }
+    // Runs `configure()` (returning a CUDA error code, 0 = ok) the first time it is called on the current device.
+    template <class F>
+    int ensure(F configure)
+    {
+        int dev = 0;
+        if (int e = device_ordinal(&dev)) return e;
+        if (dev < 0 || dev >= kMaxDevices) return configure();   // beyond the table: just set them every time
+        if (done[dev].load(std::memory_order_acquire)) return 0;
+        const int e = configure();                                 // setting twice from two threads is harmless
+        if (e == 0) done[dev].store(1, std::memory_order_release);
+        return e;
+    }
+    static int device_ordinal(int *dev);   // api.cu (cudaGetDevice)
+};
 
 // plan.cpp
 // Shared-prefix group g: `token_len[g]` consecutive tokens of the packed prefix arrays (groups back to back, in

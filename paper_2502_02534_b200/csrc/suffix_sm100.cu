@@ -270,14 +270,13 @@ int launch_one(const SuffixArgs &a, cudaStream_t st)
     using L = SuffixSmem<D>;
     static_assert(L::kTotal >= int(sizeof(float)) * kWarps * G * (D + 2), "combine buffer must fit in the ring");
     auto kern = suffix_kernel<D, G>;
-    static bool configured = false;  // attribute set once per process and instantiation
-    if (!configured) {
+    static PerDeviceOnce once;   // per instantiation
+    const int cfg_rc = once.ensure([&] {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-        if (e != cudaSuccess) return int(e);
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return int(e);
-        configured = true;
-    }
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        return int(e);
+    });
+    if (cfg_rc != 0) return cfg_rc;
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(a.num_items);
