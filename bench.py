@@ -28,8 +28,8 @@ import psa_workloads as wl  # noqa: E402
 METRIC = "sample-tokens/sec per decode step"
 UNIT = "sample-tokens/s"
 L2_BYTES = 126e6
-# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu launch list of this very command
-# (profiles/launch_list_bench_cfg2.md).  Only valid for the kernel source it was taken with.
+# DRAM bytes (read + write) per launch of the dominant kernel, from an ncu launch list of this very command
+# (dram__bytes_read.sum + dram__bytes_write.sum).  Only valid for the kernel source it was taken with.
 NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68270655 + 16007,
                         "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "93c285341b3d3d1f"}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -303,7 +303,7 @@ def run_psa(args, cfg):
                              "t_roof_ms": t_roof_ms, "frac_of_roofline": t_roof_ms / stage_avg[name] if stage_avg[name] else None}
         kernels["merge"] = {"ms": stage_avg["merge"]}
         t_roof_step = max((abytes["prefix"] + abytes["suffix"]) / (hbm * 1e9), (aflops["prefix"] + aflops["suffix"]) / (tf * 1e12)) * 1e3
-        # CPU baseline: the oracle as it stands, on this box's host cores, one full step of the same workload
+        # CPU baseline: the oracle as it stands, on this machine's host cores, one full step of the same workload
         import oracle
         best, cores = None, 0
         for _ in range(3):

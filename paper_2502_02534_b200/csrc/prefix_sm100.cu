@@ -10,19 +10,26 @@
 // (the result is unchanged: the factor cancels between O and l), so the accumulator in
 // TMEM is almost never rescaled.
 //
-// One thread block = one work item = (kv head, up to 256 query rows, a range of keys).
-// Two shapes of block, chosen per launch from the plan:
-//   two row tiles (some item has > 128 rows), 10 warps:
-//     warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1 (thread = TMEM lane = query row)
-//     warp 8           TMA producer: Q once, then K and V tiles of 128 keys through a ring of buffers
+// One thread block = one work item = (kv head, up to 256 query rows, a range of keys); thread = TMEM lane =
+// query row.  Per key tile and row tile:  S = Q K^T (SS MMA, K-major operands, 128-byte swizzle) -> the softmax
+// warpgroup reads S from TMEM and writes P (bf16) back to TMEM -> O += P V (TS MMA, P from TMEM, V as MN-major B
+// operand).  K/V are read from HBM/L2 once per item.  Three shapes of block, chosen per launch from the plan:
+//   two row tiles (some item has > 128 rows), 10 warps, 128-key tiles, ring of 5 tiles:
+//     warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1
+//     warp 8           TMA producer: Q once, then K and V tiles through a ring of buffers
 //     warp 9           MMA issuer (one lane) and owner of the TMEM allocation
-//     The two row tiles alternate on the tensor pipe, so one tile's softmax overlaps the other's MMAs.
-//   one row tile (every item has <= 128 rows), 6 warps: warps 0-3 softmax, 4 producer, 5 MMA.
-//     The two S buffers alternate by key tile instead, so QK^T of tile j+1 runs under the softmax
-//     of tile j; the block is small enough to share an SM with a block of the suffix stage.
-// Per key tile and row tile:  S = Q K^T (SS MMA, K-major operands, 128-byte swizzle)
-// -> softmax warpgroup reads S from TMEM, writes P (bf16) over it -> O += P V (TS MMA,
-// P from TMEM, V as MN-major B operand).  K/V are read from HBM/L2 once per item.
+//     The two row tiles alternate on the tensor pipe (one tile's softmax overlaps the other's MMAs); P is written
+//     over S.  TMEM: S0 S1 at columns 0 / 128, O0 O1 at 256 / 256 + D.
+//   one row tile, small (<= 128 rows; short items, or enough rows not to be purely HBM-bound), 6 warps
+//     (0-3 softmax, 4 producer, 5 MMA), <= 144 registers, 129 KB of shared memory: ONE SUFFIX BLOCK FITS BESIDE IT
+//     on the SM.  64-key tiles through a ring of 6 (three tiles of look-ahead in 96 KB); S0/S1 alternate by key
+//     tile so that QK^T of tile j+1 runs under the softmax of tile j; P has TMEM columns of its own (384..511),
+//     which keeps S intact and makes the common softmax a single pass against the current reference maximum.
+//   one row tile, long (<= 64 rows and long items: HBM-bound): the same with 128-key tiles and a ring of 6; owns the SM.
+// The epilogue sends O / l through a padded staging tile laid over the idle ring, so that every global store
+// instruction writes one full row.  Launched as a programmatic dependent: set-up (barriers, TMEM) overlaps the
+// tail of the preceding kernel, `griddepcontrol.wait` precedes the first memory access, and the suffix stage is
+// released to run beside this grid.
 //
 // Every wait on an mbarrier is bounded: when the limit passes, the block raises
 // PSA_ERR_TIMEOUT in the status word, stops storing results, and drains to a normal exit
