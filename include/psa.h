@@ -233,6 +233,16 @@ psa_status_t psa_decode_host(const psa_plan_t *plan, const void *q_host,
 psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cuda_stream);
 
 /*
+ * Debug aid (no counterpart in the paper): check a page table against the plan before the suffix stage trusts it.
+ * For every sample: 0 <= suffix_lens[s] <= the planned bound, at least ceil(S_s / 16) pages in its list, every
+ * page id in [0, num_pool_pages).  Enqueues one small kernel; a violation raises PSA_ERR_BOUNDS in the status
+ * word of `workspace` (read it with psa_check_status).  psa_decode itself does not check page ids.
+ */
+psa_status_t psa_validate_page_table(const psa_plan_t *plan, const int32_t *page_indptr, const int32_t *page_indices,
+                                     const int32_t *suffix_lens, int64_t num_pool_pages, void *workspace,
+                                     size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The step after the path: append one new token per sample to the paged suffix K/V (each of the paper's samples
  * grows by one token per decode step, up to 1024: appendix "Experiment details").  For every sample s, the rows
  * new_k[s], new_v[s] ([B, Hkv, D] bf16 device, contiguous) are written to position S_s = suffix_lens[s] of the

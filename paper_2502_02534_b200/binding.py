@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -100,6 +100,8 @@ def library():
         lib.psa_check_status.argtypes = [P, P, P]
         lib.psa_append_kv.restype = c_int32
         lib.psa_append_kv.argtypes = [P, P, P, P, P, POINTER(c_int64), P, P, P, P, c_size_t, P]
+        lib.psa_validate_page_table.restype = c_int32
+        lib.psa_validate_page_table.argtypes = [P, P, P, P, c_int64, P, c_size_t, P]
         lib.psa_selftest_bounded_wait.restype = c_int32
         lib.psa_selftest_bounded_wait.argtypes = [P, c_size_t, ctypes.c_uint64, P]
         lib.psa_status_string.restype = c_char_p
@@ -208,6 +210,13 @@ class Plan:
         _check(library().psa_plan_bind_workspace(self._h, _ptr(workspace), workspace.numel(), _stream_ptr(stream)))
         self.workspace = workspace
         return workspace
+
+    def validate_page_table(self, page_indptr, page_indices, suffix_lens, num_pool_pages, stream=None):
+        """psa_validate_page_table: enqueue the check; check_status() raises PSA_ERR_BOUNDS if the table is bad."""
+        if self.workspace is None:
+            self.bind_workspace(stream=stream)
+        _check(library().psa_validate_page_table(self._h, _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens),
+                                                 int(num_pool_pages), _ptr(self.workspace), self.workspace.numel(), _stream_ptr(stream)))
 
     def selftest_bounded_wait(self, limit_ns=2_000_000, stream=None):
         """Enqueue the kernel whose wait can never be satisfied; check_status() must then raise PSA_ERR_TIMEOUT."""

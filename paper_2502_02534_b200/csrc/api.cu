@@ -386,6 +386,22 @@ psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void
     return PSA_OK;
 }
 
+psa_status_t psa_validate_page_table(const psa_plan_t *plan, const int32_t *page_indptr, const int32_t *page_indices,
+                                     const int32_t *suffix_lens, int64_t num_pool_pages, void *workspace,
+                                     size_t workspace_bytes, void *cuda_stream)
+{
+    Carved c;
+    psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
+    if (st != PSA_OK) return st;
+    if (!page_indptr || !suffix_lens || (!page_indices && plan->total_suffix_bound_hint() > 0))
+        return fail(PSA_ERR_INVALID_ARG, "null page table");
+    if (num_pool_pages < 0 || num_pool_pages > (int64_t(1) << 31) - 1) return fail(PSA_ERR_INVALID_ARG, "num_pool_pages out of range");
+    const int rc = psa::launch_validate(page_indptr, page_indices, suffix_lens, c.sample_info, plan->num_samples,
+                                        int(num_pool_pages), c.status, cuda_stream);
+    if (rc != 0) return cuda_fail(cudaError_t(rc), "validate launch");
+    return PSA_OK;
+}
+
 psa_status_t psa_selftest_bounded_wait(void *workspace, size_t workspace_bytes, uint64_t limit_ns, void *cuda_stream)
 {
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < sizeof(int32_t) * psa::kStatusWords)

@@ -49,7 +49,36 @@ append_kernel(const uint4 *__restrict__ new_k, const uint4 *__restrict__ new_v, 
     if (threadIdx.x == 0) suffix_lens[s] = pos + 1;
 }
 
+// Debug aid: check a page table against the plan before trusting it to the suffix stage.  One thread per sample:
+// 0 <= S_s <= planned bound, enough pages for S_s tokens, every page id inside the pool.  The first violation
+// raises PSA_ERR_BOUNDS in the status word; nothing is dereferenced beyond the tables themselves.
+__global__ void validate_kernel(const int32_t *__restrict__ page_indptr, const int32_t *__restrict__ page_indices,
+                                const int32_t *__restrict__ suffix_lens, const SampleInfo *__restrict__ sample_info,
+                                int num_samples, int num_pool_pages, int *__restrict__ status)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= num_samples) return;
+    const int S = suffix_lens[s], first = page_indptr[s], n_pages = page_indptr[s + 1] - first;
+    bool ok = S >= 0 && S <= sample_info[s].suf_len_bound && first >= 0 && n_pages >= 0 &&
+              n_pages >= (S + kPageSize - 1) / kPageSize;
+    if (ok)
+        for (int i = 0; i < (S + kPageSize - 1) / kPageSize; ++i) {
+            const int pg = page_indices[first + i];
+            ok = ok && pg >= 0 && pg < num_pool_pages;
+        }
+    if (!ok) atomicCAS(status, 0, int(PSA_ERR_BOUNDS));
+}
+
 }  // namespace
+
+int launch_validate(const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
+                    const SampleInfo *sample_info, int num_samples, int num_pool_pages, int32_t *status, void *stream)
+{
+    if (num_samples == 0) return 0;
+    validate_kernel<<<(num_samples + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        page_indptr, page_indices, suffix_lens, sample_info, num_samples, num_pool_pages, status);
+    return int(cudaGetLastError());
+}
 
 int launch_append(const AppendArgs &a, void *stream)
 {

@@ -90,6 +90,7 @@ struct psa_plan {
     int64_t num_partial_rows = 0;
     psa::WorkspaceLayout ws;
     std::vector<unsigned char> upload;  // host image of [0, ws.lists_end)
+    int64_t total_suffix_bound_hint() const { int64_t t = 0; for (int32_t v : suffix_len_bounds) t += v; return t; }
 };
 
 namespace psa {
@@ -178,5 +179,7 @@ struct AppendArgs {
     int32_t *status;
 };
 int launch_append(const AppendArgs &a, void *stream);
+int launch_validate(const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
+                    const SampleInfo *sample_info, int num_samples, int num_pool_pages, int32_t *status, void *stream);
 
 }  // namespace psa

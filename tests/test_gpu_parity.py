@@ -401,3 +401,30 @@ def test_decode_append_decode_loop_reuses_one_plan():
         plan.check_status()
     assert e.value.status == 6
     assert torch.equal(before, dev["pool_k"]) and np.array_equal(dev["suffix_lens"].cpu().numpy(), bounds)
+
+
+def test_page_table_validator_flags_bad_tables_only():
+    import torch
+    from paper_2502_02534_b200 import PsaError
+    w = wl.make_workload(cfg(samples_per_prefix=6, suffix_len=(20, 90), permute_pages=True))
+    dev = to_device(w)
+    plan = make_plan(w)
+    n_pool = w["pool_k"].shape[0]
+    plan.validate_page_table(dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], n_pool)
+    plan.check_status()                                                  # a good table passes
+    def expect_bad(indptr, indices, lens, pool=n_pool):
+        plan.validate_page_table(indptr, indices, lens, pool)
+        with pytest.raises(PsaError) as e:
+            plan.check_status()
+        assert e.value.status == 6
+    bad = dev["page_indices"].clone(); bad[3] = n_pool                   # page id outside the pool
+    expect_bad(dev["page_indptr"], bad, dev["suffix_lens"])
+    bad = dev["page_indices"].clone(); bad[0] = -1
+    expect_bad(dev["page_indptr"], bad, dev["suffix_lens"])
+    lens = dev["suffix_lens"].clone(); lens[2] += 1                      # above the planned bound
+    expect_bad(dev["page_indptr"], dev["page_indices"], lens)
+    indptr = dev["page_indptr"].clone(); indptr[1:] -= 1                 # sample 0 one page short (its length needs them all)
+    expect_bad(indptr, dev["page_indices"], dev["suffix_lens"])
+    expect_bad(dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], pool=1)
+    plan.validate_page_table(dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], n_pool)
+    plan.check_status()
