@@ -205,7 +205,7 @@ def run_psa(args, cfg):
     torch.cuda.synchronize()
 
     # ---- a decode step is launch-bound on the host (three tiny kernels), so the timed loop replays CUDA
-    # graphs, one captured step per input copy, as a serving loop would
+    # graphs of several captured steps, as a serving loop would
     def capture(fn, count):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
