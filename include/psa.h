@@ -114,6 +114,21 @@ psa_status_t psa_plan_create(const psa_config_t *cfg, int32_t num_prefixes,
 psa_status_t psa_plan_create_cascade(const psa_config_t *cfg, int32_t num_groups, const int32_t *group_first_sample,
                                      const int32_t *group_n_samples, const int32_t *group_token_len, int32_t num_samples,
                                      const int32_t *suffix_lens, psa_plan_t **out_plan);
+/*
+ * The step before the path: prefill, i.e. causal attention of a prompt over itself (token i attends to tokens
+ * 0..i of its prompt), which a decoder runs once per prompt before the samples share the resulting K/V -- and
+ * again when demonstrations are added between iterations (section "Stratification and selection").  The same
+ * tensor-core kernel serves it: every query token is a row, the 256 / G tokens of a row group share the keys up
+ * to the group's last token, and the kernel masks the keys beyond each row's own token.
+ *   prompt_lens [num_prompts] host.  Prompts are packed back to back in q / k / v / out / lse.
+ * psa_prefill: q [T, Hq, D] bf16, k / v bf16 with element (token t, kv head, d) at t*kv_strides[0] +
+ * head*kv_strides[1] + d, out [T, Hq, D] (bf16 or f32 per cfg.out_dtype), lse [T, Hq] f32; T = sum of prompt_lens;
+ * all device memory; workspace bound with psa_plan_bind_workspace.  Only enqueues work.
+ */
+psa_status_t psa_plan_create_prefill(const psa_config_t *cfg, int32_t num_prompts, const int32_t *prompt_lens,
+                                     psa_plan_t **out_plan);
+psa_status_t psa_prefill(const psa_plan_t *plan, const void *q, const void *k, const void *v, const int64_t kv_strides[2],
+                         void *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream);
 psa_status_t psa_plan_destroy(psa_plan_t *plan);
 psa_status_t psa_plan_get_info(const psa_plan_t *plan, psa_plan_info_t *info);
 

@@ -172,3 +172,31 @@ def append_kv(w: dict, new_k: np.ndarray, new_v: np.ndarray) -> dict:
         lens[s] = S + 1
     out["suffix_lens"] = lens
     return out
+
+
+def causal_attend(q, k, v, prompt_lens, sm_scale, rows=None, n_threads: int = 0):
+    """Prefill: causal self-attention of packed prompts.  q [T, Hq, D], k / v [T, Hkv, D] as bf16 bits (uint16).
+    Returns (out [n_rows, D], lse [n_rows]) in float64; rows = token * Hq + head."""
+    lib = _load()
+    lib.psa_oracle_causal.restype = ctypes.c_int
+    lib.psa_oracle_causal.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+    q, k, v = (np.ascontiguousarray(a) for a in (q, k, v))
+    assert q.dtype == np.uint16 and k.dtype == np.uint16 and v.dtype == np.uint16
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    lens = _c(prompt_lens, np.int32)
+    assert int(lens.sum()) == T == k.shape[0] == v.shape[0]
+    if rows is None:
+        n_rows, rows_ptr = T * Hq, None
+    else:
+        rows = _c(rows, np.int64)
+        n_rows, rows_ptr = len(rows), rows.ctypes.data
+    out = np.zeros((n_rows, D), dtype=np.float64)
+    lse = np.zeros((n_rows,), dtype=np.float64)
+    rc = lib.psa_oracle_causal(len(lens), lens.ctypes.data, Hq, Hkv, D, float(sm_scale), q.ctypes.data, k.ctypes.data,
+                               v.ctypes.data, rows_ptr, n_rows, out.ctypes.data, lse.ctypes.data, int(n_threads))
+    if rc != 0:
+        raise RuntimeError("psa_oracle_causal failed")
+    return out, lse

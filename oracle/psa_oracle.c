@@ -200,3 +200,60 @@ int64_t psa_oracle_weights(const psa_oracle_problem *pb, int s, int h, double *w
     free(x); free(o);
     return n;
 }
+
+/*
+ * The step before the path: causal self-attention of packed prompts (prefill).  Token i of a prompt attends to
+ * tokens 0..i of the same prompt; otherwise exactly the operator above (same scale, same GQA mapping, same two
+ * passes).  q is [T, Hq, D], k and v are [T, Hkv, D] bf16 bit patterns, prompts packed back to back;
+ * rows[i] = token * Hq + head (NULL = all), out [n_rows, D], lse [n_rows].
+ */
+int psa_oracle_causal(int num_prompts, const int32_t *prompt_lens, int num_q_heads, int num_kv_heads, int head_dim,
+                      double sm_scale, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                      const int64_t *rows, int64_t n_rows, double *out, double *lse, int n_threads)
+{
+    int64_t T = 0, maxL = 1;
+    for (int p = 0; p < num_prompts; ++p) { T += prompt_lens[p]; if (prompt_lens[p] > maxL) maxL = prompt_lens[p]; }
+    if (rows == NULL) n_rows = T * num_q_heads;
+    const int D = head_dim, G = num_q_heads / num_kv_heads;
+    int failed = 0;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#pragma omp parallel
+#endif
+    {
+        double *x = (double *)malloc(sizeof(double) * (size_t)maxL);
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+        for (int64_t i = 0; i < n_rows; ++i) {
+            const int64_t r = rows ? rows[i] : i;
+            if (!x || r < 0 || r >= T * num_q_heads) { failed = 1; continue; }
+            const int64_t tok = r / num_q_heads;
+            const int h = (int)(r % num_q_heads), kv = h / G;
+            int64_t first = 0;                       /* first token of the prompt that holds `tok` */
+            for (int p = 0; p < num_prompts; ++p) { if (tok < first + prompt_lens[p]) break; first += prompt_lens[p]; }
+            const int64_t n = tok - first + 1;       /* the token's own key is the last one it sees */
+            const uint16_t *qrow = q + (tok * num_q_heads + h) * D;
+            double m = -INFINITY, Z = 0.0;
+            for (int64_t j = 0; j < n; ++j) {
+                const uint16_t *krow = k + ((first + j) * num_kv_heads + kv) * D;
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+                x[j] = sm_scale * dot;
+                if (x[j] > m) m = x[j];
+            }
+            double *o = out + i * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            for (int64_t j = 0; j < n; ++j) {
+                const uint16_t *vrow = v + ((first + j) * num_kv_heads + kv) * D;
+                const double w = exp(x[j] - m);
+                Z += w;
+                for (int d = 0; d < D; ++d) o[d] += w * bf16_to_f64(vrow[d]);
+            }
+            for (int d = 0; d < D; ++d) o[d] /= Z;
+            lse[i] = m + log(Z);
+        }
+        free(x);
+    }
+    return failed ? -1 : 0;
+}

@@ -15,7 +15,7 @@ PSA_OUT_BF16, PSA_OUT_F32 = 0, 1
 
 # every symbol include/psa.h declares
 EXPORTED_SYMBOLS = [
-    "psa_plan_create", "psa_plan_create_cascade", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
+    "psa_plan_create", "psa_plan_create_cascade", "psa_plan_create_prefill", "psa_prefill", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
     "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table",
@@ -70,6 +70,10 @@ def library():
         lib.psa_plan_create.argtypes = [POINTER(_Config), c_int32, P, P, P, POINTER(c_void_p)]
         lib.psa_plan_create_cascade.restype = c_int32
         lib.psa_plan_create_cascade.argtypes = [POINTER(_Config), c_int32, P, P, P, c_int32, P, POINTER(c_void_p)]
+        lib.psa_plan_create_prefill.restype = c_int32
+        lib.psa_plan_create_prefill.argtypes = [POINTER(_Config), c_int32, P, POINTER(c_void_p)]
+        lib.psa_prefill.restype = c_int32
+        lib.psa_prefill.argtypes = [P, P, P, P, POINTER(c_int64), P, P, P, c_size_t, P]
         lib.psa_plan_destroy.restype = c_int32
         lib.psa_plan_destroy.argtypes = [P]
         lib.psa_plan_get_info.restype = c_int32
@@ -148,7 +152,7 @@ class Plan:
 
     def __init__(self, prefix_lens, n_samples_per_prefix, suffix_lens, *, num_q_heads, num_kv_heads, head_dim,
                  page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0, suffix_chunk_tokens=0, prefix_tiles_per_item=0,
-                 prefix_rows_per_item=0, groups=None):
+                 prefix_rows_per_item=0, groups=None, prefill_prompt_lens=None):
         """``groups`` = (first_sample[], n_samples[], token_len[]) plans a cascade of shared prefixes
         (psa_plan_create_cascade); ``prefix_lens`` / ``n_samples_per_prefix`` are then ignored."""
         lib = library()
@@ -160,7 +164,10 @@ class Plan:
                       suffix_chunk_tokens, prefix_tiles_per_item, prefix_rows_per_item, 0)
         handle = c_void_p()
         self._h = None
-        if groups is None:
+        if prefill_prompt_lens is not None:     # causal self-attention of whole prompts (psa_plan_create_prefill)
+            self.prompt_lens = _i32(prefill_prompt_lens)
+            _check(lib.psa_plan_create_prefill(ctypes.byref(cfg), len(self.prompt_lens), _ptr(self.prompt_lens), ctypes.byref(handle)))
+        elif groups is None:
             _check(lib.psa_plan_create(ctypes.byref(cfg), len(self.prefix_lens), _ptr(self.prefix_lens), _ptr(self.n_samples),
                                        _ptr(self.suffix_len_bounds), ctypes.byref(handle)))
         else:
@@ -276,6 +283,15 @@ def decode_static(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_poo
     _check(library().psa_decode_static(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, _ptr(suffix_k_pool),
                                        _ptr(suffix_v_pool), qst, _ptr(page_indptr), _ptr(page_indices),
                                        _ptr(suffix_lens), _ptr(out), _ptr(lse), _stream_ptr(stream)))
+
+
+def prefill(plan: Plan, q, k, v, out, lse, *, kv_strides=None, stream=None):
+    """psa_prefill on torch CUDA tensors: causal attention of every prompt over itself."""
+    if plan.workspace is None:
+        plan.bind_workspace(stream=stream)
+    st = _strides(kv_strides or default_prefix_strides(plan), 2)
+    _check(library().psa_prefill(plan.handle, _ptr(q), _ptr(k), _ptr(v), st, _ptr(out), _ptr(lse), _ptr(plan.workspace),
+                                 plan.workspace.numel(), _stream_ptr(stream)))
 
 
 def append_kv(plan: Plan, new_k, new_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens, *,

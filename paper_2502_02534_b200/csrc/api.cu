@@ -1,6 +1,7 @@
 // C ABI of the library (include/psa.h): argument checks, workspace carving, stage launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstring>
 #include <new>
 #include <string>
@@ -58,7 +59,8 @@ extern "C" {
 
 static psa_status_t create_impl(const psa_config_t *cfg, int32_t num_groups, const int32_t *first_sample,
                                 const int32_t *n_samples, const int32_t *token_len, int32_t num_samples,
-                                const int32_t *suffix_lens, psa_plan_t **out_plan)
+                                const int32_t *suffix_lens, psa_plan_t **out_plan, const int32_t *token_begin = nullptr,
+                                int64_t total_tokens = 0, bool causal = false)
 {
     if (!cfg || !out_plan) return fail(PSA_ERR_INVALID_ARG, "null cfg or out_plan");
     *out_plan = nullptr;
@@ -73,7 +75,8 @@ static psa_status_t create_impl(const psa_config_t *cfg, int32_t num_groups, con
     psa_plan *plan = new (std::nothrow) psa_plan();
     if (!plan) return fail(PSA_ERR_INVALID_ARG, "out of host memory");
     std::string err;
-    psa_status_t st = psa::build_plan(c, num_groups, first_sample, n_samples, token_len, num_samples, suffix_lens, plan, &err);
+    psa_status_t st = psa::build_plan(c, num_groups, first_sample, n_samples, token_len, token_begin, total_tokens, causal, num_samples,
+                                      suffix_lens, plan, &err);
     if (st != PSA_OK) {
         delete plan;
         return fail(st, err);
@@ -103,6 +106,40 @@ psa_status_t psa_plan_create_cascade(const psa_config_t *cfg, int32_t num_groups
                                      const int32_t *suffix_lens, psa_plan_t **out_plan)
 {
     return create_impl(cfg, num_groups, group_first_sample, group_n_samples, group_token_len, num_samples, suffix_lens, out_plan);
+}
+
+psa_status_t psa_plan_create_prefill(const psa_config_t *cfg, int32_t num_prompts, const int32_t *prompt_lens,
+                                     psa_plan_t **out_plan)
+{
+    if (!cfg || !out_plan) return fail(PSA_ERR_INVALID_ARG, "null cfg or out_plan");
+    if (num_prompts < 0 || (num_prompts > 0 && !prompt_lens)) return fail(PSA_ERR_INVALID_ARG, "null prompt_lens");
+    if (cfg->num_kv_heads <= 0 || cfg->num_q_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads)
+        return fail(PSA_ERR_INVALID_ARG, "num_q_heads must be a positive multiple of num_kv_heads");
+    const int G = cfg->num_q_heads / cfg->num_kv_heads;
+    if (G > 8) return fail(PSA_ERR_UNSUPPORTED, "group size must be 1, 2, 4 or 8");
+    // Every query token is a "sample" without a suffix.  The tokens of one row group (256 query rows = 256 / G
+    // tokens) form a prefix group whose keys are the prompt's tokens up to the group's last token; the causal
+    // mask inside the kernel trims the diagonal.
+    const int tokens_per_group = psa::kPrefixRowsPerItem / G;
+    std::vector<int32_t> first, count, len, begin;
+    int64_t total = 0;
+    for (int32_t p = 0; p < num_prompts; ++p) {
+        if (prompt_lens[p] < 0) return fail(PSA_ERR_INVALID_ARG, "negative prompt length");
+        for (int64_t t0 = 0; t0 < prompt_lens[p]; t0 += tokens_per_group) {
+            const int64_t n = std::min<int64_t>(tokens_per_group, prompt_lens[p] - t0);
+            first.push_back(int32_t(total + t0));
+            count.push_back(int32_t(n));
+            len.push_back(int32_t(t0 + n));
+            begin.push_back(int32_t(total));
+        }
+        total += prompt_lens[p];
+        if (total > (1 << 24)) return fail(PSA_ERR_UNSUPPORTED, "problem too large");
+    }
+    std::vector<int32_t> zero_suffix(size_t(total), 0);
+    psa_config_t c = *cfg;
+    if (c.prefix_rows_per_item == 0) c.prefix_rows_per_item = psa::kPrefixRowsPerItem;
+    return create_impl(&c, int32_t(first.size()), first.data(), count.data(), len.data(), int32_t(total), zero_suffix.data(),
+                       out_plan, begin.data(), total, true);
 }
 
 psa_status_t psa_plan_destroy(psa_plan_t *plan)
@@ -177,6 +214,7 @@ psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void
     a.sm_scale = plan->cfg.sm_scale;
     a.items = c.prefix_items; a.num_items = int32_t(plan->prefix_items.size());
     a.max_rows_per_item = plan->prefix_max_rows_per_item; a.max_tiles_per_item = plan->prefix_tiles_per_item;
+    a.causal = plan->causal;
     a.partial_o = c.partial_o; a.partial_lse = c.partial_lse; a.status = c.status;
     std::string err;
     if (psa::launch_prefix(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
@@ -247,6 +285,19 @@ psa_status_t psa_decode_merge(const psa_plan_t *plan, const int32_t *suffix_lens
                               size_t workspace_bytes, void *cuda_stream)
 {
     return merge_impl(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream, false);
+}
+
+psa_status_t psa_prefill(const psa_plan_t *plan, const void *q, const void *k, const void *v, const int64_t kv_strides[2],
+                         void *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Carved c;
+    psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
+    if (st != PSA_OK) return st;
+    if (!plan->causal) return fail(PSA_ERR_INVALID_ARG, "psa_prefill needs a plan made by psa_plan_create_prefill");
+    st = psa_decode_prefix(plan, q, k, v, kv_strides, workspace, workspace_bytes, cuda_stream);
+    if (st != PSA_OK) return st;
+    const int32_t *zero_lens = reinterpret_cast<const int32_t *>(static_cast<unsigned char *>(workspace) + plan->ws.zero_lens_off);
+    return merge_impl(plan, zero_lens, out, lse, workspace, workspace_bytes, cuda_stream, !plan->prefix_items.empty());
 }
 
 psa_status_t psa_decode(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,

@@ -79,8 +79,8 @@ int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sm
 }  // namespace
 
 psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first_sample, const int32_t *n_samples,
-                        const int32_t *prefix_lens, int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan,
-                        std::string *err)
+                        const int32_t *prefix_lens, const int32_t *token_begin, int64_t total_tokens_arg, bool causal,
+                        int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan, std::string *err)
 {
     auto fail = [&](psa_status_t st, const char *msg) { if (err) *err = msg; return st; };
     if (cfg.num_q_heads <= 0 || cfg.num_kv_heads <= 0 || cfg.num_q_heads % cfg.num_kv_heads != 0)
@@ -104,6 +104,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     if (num_samples < 0) return fail(PSA_ERR_INVALID_ARG, "negative sample count");
 
     plan->cfg = cfg;
+    plan->causal = causal;
     plan->group = G;
     plan->num_prefixes = P;
     plan->group_first_sample.assign(first_sample, first_sample + P);
@@ -116,6 +117,12 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
         if (first_sample[p] < 0 || int64_t(first_sample[p]) + n_samples[p] > B)
             return fail(PSA_ERR_INVALID_ARG, "a prefix group reaches outside the samples");
         total_tokens += prefix_lens[p];
+    }
+    if (token_begin) {   // explicit key ranges (they may overlap): the caller says how long the packed arrays are
+        total_tokens = total_tokens_arg;
+        for (int p = 0; p < P; ++p)
+            if (token_begin[p] < 0 || int64_t(token_begin[p]) + prefix_lens[p] > total_tokens)
+                return fail(PSA_ERR_INVALID_ARG, "a prefix group reaches outside the packed prefix arrays");
     }
     if (B > (1 << 24) || total_tokens > (int64_t(1) << 30)) return fail(PSA_ERR_UNSUPPORTED, "problem too large");
     if (B > 0 && !suffix_lens) return fail(PSA_ERR_INVALID_ARG, "null suffix_lens");
@@ -153,6 +160,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     int longest_item_tiles = 0;
     for (int p = 0; p < P; ++p) {
         const int64_t N = n_samples[p], L = prefix_lens[p], R = N * G, samp_off = first_sample[p];
+        if (token_begin) tok_off = token_begin[p];
         const int64_t splits = tiles[p] > 0 ? ceil_div(tiles[p], T) : 0;
         const int64_t base = next_row;
         for (int64_t i = 0; splits > 0 && i < N; ++i) {
@@ -241,6 +249,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     ws.prefix_items_off = off;    off = align_up(off + sizeof(PrefixItem) * plan->prefix_items.size(), 256);
     ws.suffix_items_off = off;    off = align_up(off + sizeof(SuffixItem) * plan->suffix_items.size(), 256);
     ws.sample_info_off = off;     off = align_up(off + sizeof(SampleInfo) * plan->sample_info.size(), 256);
+    ws.zero_lens_off = off;       off = align_up(off + (causal ? sizeof(int32_t) * size_t(B) : 0), 256);
     ws.lists_end = off;
     ws.partial_lse_off = off;     off = align_up(off + sizeof(float) * size_t(next_row), 256);
     ws.partial_o_off = off;       off = align_up(off + sizeof(float) * size_t(next_row) * size_t(cfg.head_dim), 256);

@@ -31,6 +31,12 @@
 // tail of the preceding kernel, `griddepcontrol.wait` precedes the first memory access, and the suffix stage is
 // released to run beside this grid.
 //
+// Causal mode (prefill: the "samples" of an item are consecutive prompt tokens, its keys the prompt up to the
+// item's last token): row r sees key c only if c's packed token index <= the row's own, a per-row bound on the
+// valid keys of a tile, so only an item's diagonal tiles leave the unmasked fast path.  A row that has seen no
+// key yet keeps m = -inf, l = 0; exponents are taken against 0 instead of -inf, and l = 0 ends as out = 0,
+// lse = -inf, which the merge stage ignores.
+//
 // Every wait on an mbarrier is bounded: when the limit passes, the block raises
 // PSA_ERR_TIMEOUT in the status word, stops storing results, and drains to a normal exit
 // (TMEM freed) instead of spinning.
@@ -234,7 +240,7 @@ struct PrefixSmem {
 template <int D, bool kTwo, bool kLowReg>
 __device__ __forceinline__ void
 prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensorMap *pmap_v,
-            const PrefixItem *__restrict__ items, int group, float scale_log2,
+            const PrefixItem *__restrict__ items, int group, int causal, float scale_log2,
             float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
     constexpr int kKeys = prefix_tile_keys<kLowReg>();   // keys per tile
@@ -405,7 +411,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             const uint32_t s_addr = tmem_base + lane_addr + kColS + b * 128;
             if (!(ok = mbar_wait(bar_s(b), sphase(j), abort_flag))) break;
             tc_fence_after();
-            const int valid = n_keys - j * kKeys;   // >= 1; < kKeys only on the last tile
+            // keys of this tile the row may see: all that exist (< kKeys only on the last tile) and, under the causal
+            // mask of a prefill, only those up to the row's own token (rows and keys share the packed token index)
+            int valid = n_keys - j * kKeys;
+            if (causal) valid = min(valid, first_sample + (t * kPrefixTileRows + row) / group - (first_token + j * kKeys) + 1);
 
             // Rescale the accumulator in TMEM by 2^(m_ref - m_new) for the rows whose reference maximum moves.
             // The whole warp comes here together because TMEM loads and stores are warp-collective.
@@ -456,12 +465,13 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 if (__any_sync(0xffffffffu, need)) {
                     if (!(ok = move_reference(need, tmax))) break;
                 }
+                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // a row that has seen no key yet: p = 2^(-inf) = 0
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_ref));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_ref));
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_use));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_use));
                         ps[(i >> 1) & 3] += p0 + p1;
                         sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
                     }
@@ -475,6 +485,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 // after moving the reference.  S is streamed 32 columns at a time (two chunks in flight).
                 const uint32_t p_addr = tmem_base + lane_addr + kColP + b * 64;
                 auto exp_pass = [&](float &xmax) {
+                    const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // no key seen yet: exponentiate against 0
                     uint32_t r[2][32];
                     float mx[2] = {-INFINITY, -INFINITY};
                     ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
@@ -486,8 +497,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_ref);
-                            float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_ref);
+                            float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_use);
+                            float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_use);
                             if (valid < kKeys) {   // masked keys of a ragged last tile
                                 if (c * 32 + i >= valid) x0 = -INFINITY;
                                 if (c * 32 + i + 1 >= valid) x1 = -INFINITY;
@@ -507,7 +518,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 if (j > 0) {
                     float xmax;
                     exp_pass(xmax);
-                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold);
+                    // also redo when a row meets its first visible key (its reference maximum is still -inf)
+                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold || (m_ref == -INFINITY && xmax != -INFINITY));
                 }
                 if (redo) {
                     // the tile's maximum, then the classic update, then the exponentials again
@@ -543,7 +555,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         float *stage = reinterpret_cast<float *>(smem + L::kRingOff + t * L::kStageBytes);
         if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l_sum;
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;   // a row that saw no key in this item: O = 0, lse = -inf
             float *mine = stage + row * L::kStageRowFloats;
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
@@ -557,7 +569,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                                     __uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
             }
             const int r = t * kPrefixTileRows + row;
-            if (r < n_rows) partial_lse[prow0 + r] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+            if (r < n_rows) partial_lse[prow0 + r] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
         }
         // the four warps of this row tile meet (named barrier 1 + t), then write rows round-robin
         asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
@@ -594,10 +606,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 template <int D>
 __global__ void __launch_bounds__(320, 1)
 prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
                   float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
 }
 
 // At most 144 registers per thread: two of these warps and one suffix warp (208) fit the 512 registers per lane of
@@ -605,20 +617,20 @@ prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 template <int D>
 __global__ void __maxnreg__(144)
 prefix_kernel_one(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
+                  const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
                   float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
 }
 
 // One row tile, long items: the block owns the SM anyway (long ring), so S stays in registers.
 template <int D>
 __global__ void __launch_bounds__(192, 1)
 prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group,
+                       const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
                        float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
 {
-    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
 }
 
 // Self-test of the bounded wait: one block waits on a barrier that nothing ever arrives on.  The wait must give
@@ -703,7 +715,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     attr.val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = &attr;
     lc.numAttrs = 1;   // set-up may overlap the tail of the preceding kernel; the kernel waits before touching memory
-    return int(cudaLaunchKernelEx(&lc, kern, mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, scale_log2, a.partial_o,
+    return int(cudaLaunchKernelEx(&lc, kern, mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, int(a.causal), scale_log2, a.partial_o,
                                   a.partial_lse, a.status));
 }
 

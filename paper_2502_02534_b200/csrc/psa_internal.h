@@ -66,6 +66,7 @@ struct WorkspaceLayout {
     size_t prefix_items_off = 0;
     size_t suffix_items_off = 0;
     size_t sample_info_off = 0;
+    size_t zero_lens_off = 0;     // int32 [B] of zeros: the suffix lengths of a prefill plan
     size_t lists_end = 0;        // bytes copied by bind_workspace
     size_t partial_lse_off = 0;  // float [num_partial_rows]
     size_t partial_o_off = 0;    // float [num_partial_rows, D]
@@ -86,6 +87,7 @@ struct psa_plan {
     std::vector<psa::SampleInfo> sample_info;
     int32_t prefix_tiles_per_item = 0;
     int32_t prefix_max_rows_per_item = 0;
+    bool causal = false;          // a prefill plan
     int32_t suffix_chunk_tokens = 0;
     int64_t num_partial_rows = 0;
     psa::WorkspaceLayout ws;
@@ -122,9 +124,11 @@ struct PerDeviceOnce {
 // plan.cpp
 // Shared-prefix group g: `token_len[g]` consecutive tokens of the packed prefix arrays (groups back to back, in
 // order) attended by samples [first_sample[g], first_sample[g] + n_samples[g]).
+// token_begin == nullptr: group g starts where group g-1 ends.  causal: keys beyond a row's own packed token index
+// are masked (prefill: "samples" are the prompt's tokens).
 psa_status_t build_plan(const psa_config_t &cfg, int32_t num_groups, const int32_t *first_sample, const int32_t *n_samples,
-                        const int32_t *token_len, int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan,
-                        std::string *err);
+                        const int32_t *token_len, const int32_t *token_begin, int64_t total_tokens, bool causal,
+                        int32_t num_samples, const int32_t *suffix_lens, psa_plan *plan, std::string *err);
 
 // Launchers (one per .cu file). All enqueue on `stream` and return a CUDA error code (0 = ok).
 struct PrefixArgs {
@@ -136,6 +140,7 @@ struct PrefixArgs {
     const PrefixItem *items;  // device
     int32_t num_items;
     int32_t max_rows_per_item, max_tiles_per_item;  // over all items of the plan
+    bool causal = false;  // prefill: row (token) i sees keys up to its own packed token index
     float *partial_o, *partial_lse;  // device
     int32_t *status;                 // device
 };

@@ -387,3 +387,51 @@ def test_append_puts_the_new_token_last_in_every_context():
     with pytest.raises(IndexError):
         w3 = dict(w); w3["suffix_lens"] = (np.array(w["page_indptr"][1:]) - np.array(w["page_indptr"][:-1])) * 4
         oracle.append_kv(w3, new_k, new_v)
+
+
+# ---------------------------------------------------------------- prefill (causal) oracle
+def _prefill_inputs(lens, Hq=4, Hkv=2, D=8, seed=31):
+    T = int(np.sum(lens))
+    return (wl.normal_bf16((T, Hq, D), seed, 1), wl.normal_bf16((T, Hkv, D), seed, 2), wl.normal_bf16((T, Hkv, D), seed, 3))
+
+
+def test_causal_oracle_equals_the_pinned_operator_on_growing_prefixes():
+    """Token i of a prompt = one sample whose whole context is the prompt's first i+1 tokens, copied out."""
+    lens = [5, 1, 7]
+    q, k, v = _prefill_inputs(lens)
+    out, lse = oracle.causal_attend(q, k, v, lens, 0.35)
+    offs = np.concatenate([[0], np.cumsum(lens)])
+    ks, vs, plens = [], [], []
+    for p, L in enumerate(lens):
+        for i in range(L):
+            ks.append(k[offs[p]: offs[p] + i + 1]); vs.append(v[offs[p]: offs[p] + i + 1]); plens.append(i + 1)
+    T = sum(lens)
+    flat = dict(prefix_lens=np.array(plens, np.int32), n_samples=np.ones(T, np.int32), suffix_lens=np.zeros(T, np.int32),
+                num_q_heads=4, num_kv_heads=2, head_dim=8, page_size=4, sm_scale=0.35, q=q,
+                prefix_k=np.concatenate(ks), prefix_v=np.concatenate(vs),
+                pool_k=np.zeros((1, 2, 4, 8), np.uint16), pool_v=np.zeros((1, 2, 4, 8), np.uint16),
+                page_indptr=np.zeros(T + 1, np.int32), page_indices=np.zeros(0, np.int32))
+    fo, fl, _ = oracle.attend(flat)
+    assert np.allclose(out, fo, rtol=0, atol=TOL) and np.allclose(lse, fl, rtol=0, atol=TOL)
+    # the first token of every prompt sees only itself
+    for p in range(3):
+        for h in range(4):
+            r = offs[p] * 4 + h
+            assert np.array_equal(out[r], rec.bf16_bits_to_f64(v[offs[p], h // 2]))
+
+
+def test_causal_oracle_matches_torch_masked_softmax():
+    torch = pytest.importorskip("torch")
+    lens = [9]
+    q, k, v = _prefill_inputs(lens, Hq=2, Hkv=1, D=11, seed=5)
+    out, lse = oracle.causal_attend(q, k, v, lens, 0.3)
+    Q = torch.from_numpy(rec.bf16_bits_to_f64(q)); K = torch.from_numpy(rec.bf16_bits_to_f64(k))[:, 0]; V = torch.from_numpy(rec.bf16_bits_to_f64(v))[:, 0]
+    for h in range(2):
+        S = (Q[:, h] @ K.T) * 0.3
+        S = S.masked_fill(torch.triu(torch.ones(9, 9, dtype=torch.bool), diagonal=1), float("-inf"))
+        ref = torch.softmax(S, 1) @ V
+        assert np.allclose(out.reshape(9, 2, 11)[:, h], ref.numpy(), rtol=0, atol=TOL)
+        assert np.allclose(lse.reshape(9, 2)[:, h], torch.logsumexp(S, 1).numpy(), rtol=0, atol=TOL)
+    rows = np.array([3, 17, 0])
+    o2, l2 = oracle.causal_attend(q, k, v, lens, 0.3, rows=rows)
+    assert np.array_equal(o2, out[rows]) and np.array_equal(l2, lse[rows])
