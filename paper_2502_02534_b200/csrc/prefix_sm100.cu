@@ -20,8 +20,10 @@
 //     warp 9           MMA issuer (one lane) and owner of the TMEM allocation
 //     The two row tiles alternate on the tensor pipe (one tile's softmax overlaps the other's MMAs); P is written
 //     over S.  TMEM: S0 S1 at columns 0 / 128, O0 O1 at 256 / 256 + D.
-//   one row tile, small (<= 128 rows; short items, or enough rows not to be purely HBM-bound), 6 warps
-//     (0-3 softmax, 4 producer, 5 MMA), <= 144 registers, 129 KB of shared memory: ONE SUFFIX BLOCK FITS BESIDE IT
+//   one row tile, small (<= 128 rows; short items, or enough rows not to be purely HBM-bound), 7 warps
+//     (0-3 softmax, 4 producer, 5 issuer of QK^T, 6 issuer of PV: the issuing thread polls barriers and commits
+//     between batches of MMAs, a few hundred cycles of scalar code per tile during which the tensor pipe drains, so
+//     two issuers whose waits overlap each other's MMAs shorten the key-tile period), <= 144 registers, 129 KB of shared memory: ONE SUFFIX BLOCK FITS BESIDE IT
 //     on the SM.  64-key tiles through a ring of 6 (three tiles of look-ahead in 96 KB); S0/S1 alternate by key
 //     tile so that QK^T of tile j+1 runs under the softmax of tile j; P has TMEM columns of its own (384..511),
 //     which keeps S intact and makes the common softmax a single pass against the current reference maximum.
@@ -85,7 +87,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           unsigned long long limit_ns = kWaitLimitNs)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)   // the common case ends here, without reading the (slow) global timer
+        if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -127,19 +131,22 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+// D[tmem] (+)= A * B with A from shared memory (mma_ss_w) or from tensor memory (mma_ts_w), B from shared memory.
+// Shared-memory descriptors are given as (low word, high word): the one thread that issues every
+// MMA of a block keeps the high words (layout constants) in registers and derives each low word (the address) with
+// a single add, so that issuing stays far cheaper than the MMA itself.
+__device__ __forceinline__ void mma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                         uint32_t accumulate)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+__device__ __forceinline__ void mma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns: thread = lane (row), register i = column i
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
@@ -186,18 +193,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 // ---------------------------------------------------------------- descriptors
-// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte
-// offsets (all in 16-byte units), descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= uint64_t((addr >> 4) & 0x3FFFu);
-    d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= uint64_t(1) << 46;   // version
-    d |= uint64_t(2) << 61;   // SWIZZLE_128B
-    return d;
-}
+// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets (all in 16-byte units),
+// descriptor version 1, 128-byte swizzle.
+// The descriptor's two words: only the low one depends on the address, and moving the start by `bytes` adds
+// bytes / 16 to it (tiles lie in the low 256 KB of the shared window, so the 14-bit field cannot overflow).
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr, uint32_t lbo_bytes) { return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16); }
+__host__ __device__ constexpr uint32_t smem_desc_hi(uint32_t sbo_bytes) { return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29); }
 // Instruction descriptor for kind::f16: bf16 x bf16 -> f32, M = 128.
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 {
@@ -206,7 +207,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 }
 
 // Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 10 warps); otherwise one row
-// tile (one Q tile, 6 warps).
+// tile (one Q tile, 7 warps).
 constexpr int kMaxRing = 6;
 // Ring length per block shape: 5 x 32 KB beside two Q tiles, else 6 (never fewer buffers than the epilogue
 // staging tile needs).
@@ -247,7 +248,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     using L = PrefixSmem<D, kTwo, kKeys>;
     constexpr int ring = prefix_ring<D, kTwo, kLowReg>();   // K/V tile buffers in flight
     constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
-    constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
+    constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1, kMmaWarp2 = kSoftmaxWarps + 2;
     constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
     constexpr int kPSteps = kKeys / 16;   // MMA k-steps of PV
     constexpr uint32_t kIdescQK = make_idesc(kKeys, false);
@@ -326,74 +327,97 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     tma_load_3d(sbase + L::kRingOff + slot * L::kTileBytes + h * L::kHalfBytes, map, bar_full(slot), h * 64, kv, tok);
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == kMmaWarp || warp == kMmaWarp2) {
+        // ------------------------------------------------------------ MMA issuers: one lane of each of two warps
+        // A single issuing thread is a serial bottleneck: between two batches of MMAs it polls barriers and commits,
+        // a few hundred cycles of scalar code each time, during which the tensor pipe drains and idles.  With two
+        // issuers the waits of one overlap the MMAs of the other.
+        //   two row tiles: issuer 0 alone (see there)
+        //   one row tile:  issuer 0 issues every QK^T, issuer 1 every PV
         if (lane == 0) {
-            bool ok = mbar_wait(bar_q(), 0, abort_flag);
+            const int who = warp - kMmaWarp;
             auto wait_entry = [&](int e) { return mbar_wait(bar_full(e % ring), (e / ring) & 1, abort_flag); };
-            auto issue_qk = [&](int t, int j) {   // S[sbuf] = Q_t K_j^T ; K_j is ring entry 2j
-                const uint32_t qa = sbase + L::kQOff + t * L::kQTileBytes;
-                const uint32_t kb = sbase + L::kRingOff + ((2 * j) % ring) * L::kTileBytes;
-                const uint32_t d = tmem_base + kColS + sbuf(t, j) * 128;
+            constexpr uint32_t kHiK = smem_desc_hi(1024), kHiV = smem_desc_hi(1024);
+            const uint32_t q_lo = smem_desc_lo(sbase + L::kQOff, 16);
+            const uint32_t ring_k_lo = smem_desc_lo(sbase + L::kRingOff, 16);            // K tiles: K-major, no leading offset
+            const uint32_t ring_v_lo = smem_desc_lo(sbase + L::kRingOff, L::kHalfBytes); // V tiles: MN-major, halves kHalfBytes apart
+            auto issue_qk = [&](int t, int sb, int kslot) {   // S[sb] = Q_t K^T, K in ring slot `kslot`
+                const uint32_t a_lo = q_lo + uint32_t(t) * (L::kQTileBytes >> 4);
+                const uint32_t b_lo = ring_k_lo + uint32_t(kslot) * (L::kTileBytes >> 4);
+                const uint32_t d = tmem_base + kColS + uint32_t(sb) * 128;
 #pragma unroll
-                for (int k = 0; k < kKSteps; ++k) {
-                    mma_ss(d, make_smem_desc(qa + (k / 4) * L::kQHalfBytes + (k % 4) * 32, 16, 1024),
-                           make_smem_desc(kb + (k / 4) * L::kHalfBytes + (k % 4) * 32, 16, 1024), kIdescQK, k > 0);
-                }
+                for (int k = 0; k < kKSteps; ++k)
+                    mma_ss_w(d, a_lo + (((k / 4) * L::kQHalfBytes + (k % 4) * 32) >> 4), kHiK,
+                             b_lo + (((k / 4) * L::kHalfBytes + (k % 4) * 32) >> 4), kHiK, kIdescQK, k > 0);
             };
-            auto issue_pv = [&](int t, int j) {   // O_t += P[sbuf] V_j ; V_j is ring entry 2j+1
-                const uint32_t vb = sbase + L::kRingOff + ((2 * j + 1) % ring) * L::kTileBytes;
-                const uint32_t a = kTwo ? tmem_base + kColS + t * 128   // P over S
-                                        : tmem_base + kColP + (j & 1) * 64;
+            auto issue_pv = [&](int t, uint32_t p_tmem, int vslot, bool first) {   // O_t += P V, V in ring slot `vslot`
+                const uint32_t b_lo = ring_v_lo + uint32_t(vslot) * (L::kTileBytes >> 4);
 #pragma unroll
                 for (int k = 0; k < kPSteps; ++k)
-                    mma_ts(tmem_base + kColO + t * D, a + k * 8, make_smem_desc(vb + k * 2048, L::kHalfBytes, 1024), kIdescPV,
-                           (j > 0 || k > 0));
+                    mma_ts_w(tmem_base + kColO + t * D, p_tmem + k * 8, b_lo + ((k * 2048) >> 4), kHiV, kIdescPV, (!first || k > 0));
             };
+            auto next_slot = [&](int sl, int by) { sl += by; return sl >= ring ? sl - ring : sl; };
             if constexpr (kTwo) {
-                if (ok) ok = wait_entry(0);
+                // Two row tiles: ONE issuer, which alternates between the tiles (two threads issuing into the same
+                // pipe measured slower here: 95 us instead of 77 us on 2048 rows x 8192 keys x 8 heads).
+                bool ok = who == 0;
+                if (ok) ok = mbar_wait(bar_q(), 0, abort_flag);
+                if (ok) ok = wait_entry(0);   // K_0
                 if (ok) {
                     tc_fence_after();
-                    for (int t = 0; t < n_rt; ++t) { issue_qk(t, 0); tc_commit(bar_s(t)); }
+                    for (int t = 0; t < n_rt; ++t) { issue_qk(t, t, 0); tc_commit(bar_s(t)); }
                     tc_commit(bar_empty(0));                       // K_0 is free once both QK^T are done
                 }
+                int vslot = 1;   // ring slot of V_j; K_{j+1} is in the next one
                 for (int j = 0; ok && j < n_tiles; ++j) {
-                    if (!(ok = wait_entry(2 * j + 1))) break;
-                    if (j + 1 < n_tiles && !(ok = wait_entry(2 * j + 2))) break;
+                    const int kslot = next_slot(vslot, 1);
+                    if (!(ok = wait_entry(2 * j + 1))) break;                       // V_j
+                    if (j + 1 < n_tiles && !(ok = wait_entry(2 * j + 2))) break;    // K_{j+1}
                     for (int t = 0; t < n_rt; ++t) {
                         if (!(ok = mbar_wait(bar_p(t), sphase(j), abort_flag))) break;
                         tc_fence_after();
-                        issue_pv(t, j);
-                        if (t == n_rt - 1) tc_commit(bar_empty((2 * j + 1) % ring));
+                        issue_pv(t, tmem_base + kColS + t * 128 /* P over S */, vslot, j == 0);
+                        if (t == n_rt - 1) tc_commit(bar_empty(vslot));
                         if (j + 1 < n_tiles) {
-                            issue_qk(t, j + 1);
+                            issue_qk(t, t, kslot);
                             tc_commit(bar_s(t));
-                            if (t == n_rt - 1) tc_commit(bar_empty((2 * j + 2) % ring));
+                            if (t == n_rt - 1) tc_commit(bar_empty(kslot));
                         }
                     }
+                    vslot = next_slot(vslot, 2);
                 }
-            } else {
-                // one row tile: S0/S1 alternate by key tile, so QK^T of tile j+1 runs under the softmax of tile j
+            } else if (who == 0) {
+                // QK^T issuer.  S0/S1 alternate by key tile, so QK^T of tile j+1 runs under the softmax of tile j;
+                // S[j & 1] may be overwritten (by tile j+2) once the softmax of tile j has handed over its P.
+                bool ok = mbar_wait(bar_q(), 0, abort_flag);
                 for (int j = 0; ok && j < 2 && j < n_tiles; ++j) {
                     if (!(ok = wait_entry(2 * j))) break;
                     tc_fence_after();
-                    issue_qk(0, j);
+                    issue_qk(0, j & 1, (2 * j) % ring);
                     tc_commit(bar_s(j & 1));
                     tc_commit(bar_empty((2 * j) % ring));
                 }
+                int kslot = 4 % ring;   // ring slot of K_{j+2} = entry 2j+4
+                for (int j = 0; ok && j + 2 < n_tiles; ++j) {
+                    if (!(ok = wait_entry(2 * j + 4))) break;
+                    if (!(ok = mbar_wait(bar_p(j & 1), sphase(j), abort_flag))) break;
+                    tc_fence_after();
+                    issue_qk(0, j & 1, kslot);
+                    tc_commit(bar_s(j & 1));
+                    tc_commit(bar_empty(kslot));
+                    kslot = next_slot(kslot, 2);
+                }
+            } else {
+                // PV issuer
+                bool ok = true;
+                int vslot = 1 % ring;   // ring slot of V_j = entry 2j+1
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     if (!(ok = wait_entry(2 * j + 1))) break;
                     if (!(ok = mbar_wait(bar_p(j & 1), sphase(j), abort_flag))) break;
                     tc_fence_after();
-                    issue_pv(0, j);
-                    tc_commit(bar_empty((2 * j + 1) % ring));
-                    if (j + 2 < n_tiles) {
-                        if (!(ok = wait_entry(2 * j + 4))) break;
-                        tc_fence_after();
-                        issue_qk(0, j + 2);
-                        tc_commit(bar_s(j & 1));
-                        tc_commit(bar_empty((2 * j + 4) % ring));
-                    }
+                    issue_pv(0, tmem_base + kColP + (j & 1) * 64, vslot, j == 0);
+                    tc_commit(bar_empty(vslot));
+                    vslot = next_slot(vslot, 2);
                 }
             }
         }
@@ -484,6 +508,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 // largest exponent; only if that exceeds the threshold (or on the first tile) is the tile redone
                 // after moving the reference.  S is streamed 32 columns at a time (two chunks in flight).
                 const uint32_t p_addr = tmem_base + lane_addr + kColP + b * 64;
+                // P[b] was last read by the PV of tile j-2, which a different thread issues than the QK^T that made this S
+                if (j >= 2 && !(ok = mbar_wait(bar_empty((2 * j - 3) % ring), ((2 * j - 3) / ring) & 1, abort_flag))) break;
                 auto exp_pass = [&](float &xmax) {
                     const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // no key seen yet: exponentiate against 0
                     uint32_t r[2][32];
@@ -625,7 +651,7 @@ prefix_kernel_one(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
 // One row tile, long items: the block owns the SM anyway (long ring), so S stays in registers.
 template <int D>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(224, 1)
 prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
                        float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
@@ -707,7 +733,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(a.num_items);
-    lc.blockDim = dim3(kTwo ? 320 : 192);
+    lc.blockDim = dim3(kTwo ? 320 : 224);   // softmax warps, producer, one (two row tiles) or two MMA issuers
     lc.dynamicSmemBytes = L::total(ring);
     lc.stream = st;
     cudaLaunchAttribute attr{};
