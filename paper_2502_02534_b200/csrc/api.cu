@@ -193,8 +193,9 @@ int32_t psa_plan_suffix_items(const psa_plan_t *plan, int32_t *items4)
     return int32_t(plan->suffix_items.size());
 }
 
-psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,
-                               const int64_t prefix_strides[2], void *workspace, size_t workspace_bytes, void *cuda_stream)
+static psa_status_t prefix_impl(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,
+                                const int64_t prefix_strides[2], void *workspace, size_t workspace_bytes, void *cuda_stream,
+                                bool count_blocks)
 {
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
@@ -216,9 +217,17 @@ psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void
     a.max_rows_per_item = plan->prefix_max_rows_per_item; a.max_tiles_per_item = plan->prefix_tiles_per_item;
     a.causal = plan->causal;
     a.partial_o = c.partial_o; a.partial_lse = c.partial_lse; a.status = c.status;
+    a.launch_counter = count_blocks ? c.status + psa::kPrefixLaunchWord : nullptr;
+    a.done_counter = count_blocks ? c.status + psa::kPrefixDoneWord : nullptr;
     std::string err;
     if (psa::launch_prefix(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
     return PSA_OK;
+}
+
+psa_status_t psa_decode_prefix(const psa_plan_t *plan, const void *q, const void *prefix_k, const void *prefix_v,
+                               const int64_t prefix_strides[2], void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return prefix_impl(plan, q, prefix_k, prefix_v, prefix_strides, workspace, workspace_bytes, cuda_stream, false);
 }
 
 static psa_status_t suffix_impl(const psa_plan_t *plan, const void *q, const void *suffix_k_pool, const void *suffix_v_pool,
@@ -260,7 +269,7 @@ psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void
 }
 
 static psa_status_t merge_impl(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse, void *workspace,
-                               size_t workspace_bytes, void *cuda_stream, bool after_stage)
+                               size_t workspace_bytes, void *cuda_stream, bool after_stage, bool wait_for_prefix_count = false)
 {
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
@@ -276,6 +285,11 @@ static psa_status_t merge_impl(const psa_plan_t *plan, const int32_t *suffix_len
     a.chunk_tokens = plan->suffix_chunk_tokens; a.out_dtype = plan->cfg.out_dtype;
     a.out = out; a.lse = lse;
     a.after_stage = after_stage;
+    if (wait_for_prefix_count) {
+        a.prefix_counters = c.status + psa::kPrefixLaunchWord;
+        a.status = c.status;
+        a.prefix_blocks = int32_t(plan->prefix_items.size());
+    }
     std::string err;
     if (psa::launch_merge(a, cuda_stream, &err) != 0) return fail(PSA_ERR_CUDA, err);
     return PSA_OK;
@@ -306,15 +320,20 @@ psa_status_t psa_decode(const psa_plan_t *plan, const void *q, const void *prefi
                         const int32_t *suffix_lens, void *out, float *lse, void *workspace, size_t workspace_bytes,
                         void *cuda_stream)
 {
-    psa_status_t st = psa_decode_prefix(plan, q, prefix_k, prefix_v, prefix_strides, workspace, workspace_bytes, cuda_stream);
-    if (st != PSA_OK) return st;
+    if (!plan) return fail(PSA_ERR_INVALID_ARG, "null plan");
     // The suffix stage is independent of the prefix stage: launched as its programmatic dependent it runs
-    // beside it.  The merge stage needs both; the suffix blocks retire only after the prefix grid completed.
+    // beside it.  The merge stage needs both, but stream order (and the programmatic dependency) only puts it
+    // behind the suffix grid, so with both stages present the prefix blocks count themselves off in the workspace
+    // and the merge stage waits for the count.
     const bool have_prefix = !plan->prefix_items.empty(), have_suffix = !plan->suffix_items.empty();
+    psa_status_t st = prefix_impl(plan, q, prefix_k, prefix_v, prefix_strides, workspace, workspace_bytes, cuda_stream,
+                                  have_prefix && have_suffix);
+    if (st != PSA_OK) return st;
     st = suffix_impl(plan, q, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens, workspace,
                      workspace_bytes, cuda_stream, have_prefix);
     if (st != PSA_OK) return st;
-    return merge_impl(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream, have_prefix || have_suffix);
+    return merge_impl(plan, suffix_lens, out, lse, workspace, workspace_bytes, cuda_stream, have_prefix || have_suffix,
+                      have_prefix && have_suffix);
 }
 
 namespace {

@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restrict__ suffix_lens,
              const float *__restrict__ partial_o, const float *__restrict__ partial_lse,
              int num_rows, int num_q_heads, int group, int chunk_tokens, int out_is_f32,
-             void *__restrict__ out, float *__restrict__ lse_out)
+             void *__restrict__ out, float *__restrict__ lse_out, const int *prefix_counters, int prefix_blocks, int *__restrict__ status)
 {
     constexpr int V = D / 32;  // floats per lane: 2 or 4
     // kChunk rows are fetched together (registers: kChunk float4 per lane)
@@ -64,6 +64,32 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
         return r;
     };
 
+    // In a fused step that has both stages the preceding grid is the suffix stage, which ran beside the prefix
+    // stage; prefix blocks count themselves off after storing their results (launches x blocks in total, both
+    // counters wrap together).  The launch was announced before the suffix grid could start and every prefix block
+    // was running before the first suffix block, so the count is complete or about to be; the wait is bounded all
+    // the same.  It sits BEFORE the wait for the suffix grid, off the critical path.
+    if (prefix_blocks > 0) {
+        int lag = 0;
+        if (lane == 0) {
+            unsigned long long t0 = 0;
+            for (uint32_t spins = 0;; ++spins) {
+                // both words in one load (they are adjacent and 8-byte aligned): launches in the low half, blocks done in the high half
+                unsigned long long both;
+                asm volatile("ld.acquire.gpu.global.b64 %0, [%1];" : "=l"(both) : "l"(prefix_counters) : "memory");
+                lag = int(uint32_t(both) * uint32_t(prefix_blocks) - uint32_t(both >> 32));
+                if (lag <= 0) break;
+                if ((spins & 255u) == 255u) {
+                    unsigned long long now;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > 2000000000ull) { atomicCAS(status, 0, int(PSA_ERR_TIMEOUT)); break; }
+                }
+            }
+        }
+        lag = __shfl_sync(0xffffffffu, lag, 0);
+        if (lag > 0) return;   // timed out: the row stays unwritten, the status word says why
+    }
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // the next kernel in the stream (typically the next step's prefix stage) may set itself up meanwhile;
@@ -167,17 +193,18 @@ int launch_merge(const MergeArgs &a, void *stream, std::string *err)
     lc.attrs = &attr;
     lc.numAttrs = a.after_stage ? 1 : 0;   // start filling in while the preceding stage drains
     const int f32 = a.out_dtype == PSA_OUT_F32;
+    const int counted_blocks = (a.prefix_counters && a.status) ? a.prefix_blocks : 0;
     cudaError_t e;
     const bool small = rows <= 4096;   // few rows: latency matters, fetch 16 partial rows at a time
     if (a.head_dim == 128 && small)
         e = cudaLaunchKernelEx(&lc, merge_kernel<128, 16>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
-                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse, a.prefix_counters, counted_blocks, a.status);
     else if (a.head_dim == 128)
         e = cudaLaunchKernelEx(&lc, merge_kernel<128, 8>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
-                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse, a.prefix_counters, counted_blocks, a.status);
     else
         e = cudaLaunchKernelEx(&lc, merge_kernel<64, 16>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
-                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse);
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse, a.prefix_counters, counted_blocks, a.status);
     if (e != cudaSuccess && err) *err = std::string("merge launch: ") + cudaGetErrorString(e);
     return int(e);
 }

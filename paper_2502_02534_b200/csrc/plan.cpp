@@ -22,9 +22,14 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // group of `tiles` tiles is cut into ceil(tiles / T) items.  Items are dispatched longest first to the SMs, so
 // the stage takes about max(longest item, sum of items / SMs); every split also costs a partial result per row
 // (4*D bytes written, read again by the merge stage).  Costs are in tile steps of a one-row-tile block (~1.5 us);
-// a step of a two-row-tile block counts 1.6.  Pick the T with the smallest estimate, larger T on ties.
+// a step of a two-row-tile block counts 1.6.  In a step that also has a suffix stage the two grids run side by side
+// and the suffix stage (HBM-bound, the longer one) wants every SM, so the SM time the prefix items take is charged
+// once more at `sm_time_weight` (measured on 32 samples x 4096 + U[0,1024] tokens: 88 items of 3 tiles give a 22.2 us
+// step, 128 items of 2 tiles 23.4 us, although the prefix stage alone is faster with 128).  Pick the T with the
+// smallest estimate, larger T on ties.
 int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::vector<int64_t> &groups,
-                                 const std::vector<int64_t> &partial_rows_per_split, double step_weight, int head_dim, int num_sms)
+                                 const std::vector<int64_t> &partial_rows_per_split, double step_weight, int head_dim, int num_sms,
+                                 double sm_time_weight)
 {
     int64_t max_tiles = 0;
     for (int64_t t : tiles) max_tiles = std::max(max_tiles, t);
@@ -43,17 +48,20 @@ int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::v
             longest = std::max(longest, len);
             partial += double(partial_rows_per_split[p] * splits) * steps_per_partial_row;
         }
-        const double cost = std::max(longest, 1.1 * sum / num_sms) + partial;
+        const double cost = std::max(longest, 1.1 * sum / num_sms) + partial + sm_time_weight * sum / num_sms;
         if (cost <= best_cost) { best_cost = cost; best_T = int(T); }
     }
     return best_T;
 }
 
-// Suffix: items are dispatched greedily to 2 resident blocks per SM.  Estimate =
-// (sum of item costs) / slots + cost of one full item (the tail); cost = tokens + 384: a block
-// spends about as long finding its pages (three dependent loads) and combining its warps as it
-// spends streaming 384 tokens (measured on B200: 512-token chunks beat 128-token chunks by 30 %
-// on 32 samples x U[0,1024] tokens).
+// Suffix: items are dispatched greedily (longest first) to 2 resident blocks per SM and the stage is bound by HBM
+// as a whole, not block by block: a block alone can stream about three times its fair share of the bandwidth, so
+// one long item is no tail as long as it needs less than a third of the stage.  Estimate, in tokens streamed by
+// one slot at its fair share:
+//     max( (sum of tokens + 384 per item) / min(slots, items),  longest item / 3 + 384 ).
+// The 384 is what a block spends finding its pages (three dependent loads) and combining its warps, expressed
+// in tokens.  Measured on B200: 64 samples x U[0,2048] tokens take 41.9 us as whole-sample items (0.98 of the
+// copy bandwidth), 45.4 us in 1024-token chunks, 48.7 us in 512-token chunks.
 int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sms)
 {
     const double overhead = 384.0;
@@ -61,17 +69,19 @@ int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sm
     double best_cost = std::numeric_limits<double>::infinity();
     int best = 64;
     for (int C = 64; C <= 8192; C *= 2) {
-        double sum = 0.0;
+        double sum = 0.0, items = 0.0;
         int64_t longest = 0;
         for (int s = 0; s < n; ++s) {
             int64_t S = lens[s];
             if (S <= 0) continue;
             int64_t chunks = ceil_div(S, C);
             sum += double(num_kv_heads) * (double(S) + overhead * double(chunks));
+            items += double(num_kv_heads) * double(chunks);
             longest = std::max<int64_t>(longest, std::min<int64_t>(S, C));
         }
-        double cost = sum / slots + double(longest) + overhead;
-        if (cost < best_cost) { best_cost = cost; best = C; }
+        if (items == 0.0) break;
+        const double cost = std::max(sum / std::min(slots, items), double(longest) / 3.0 + overhead);
+        if (cost < best_cost * 0.999) { best_cost = cost; best = C; }
     }
     return best;
 }
@@ -141,6 +151,8 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     const int rows_per_item = cfg.prefix_rows_per_item > 0 ? cfg.prefix_rows_per_item
                                                            : (max_rows >= 2 * kPrefixRowsPerItem ? kPrefixRowsPerItem : kPrefixTileRows);
     const int samples_per_group = rows_per_item / G;
+    bool any_suffix = false;
+    for (int64_t s = 0; s < B; ++s) any_suffix = any_suffix || suffix_lens[s] > 0;
     std::vector<int64_t> tiles(P), groups(P), rows_per_split(P);
     for (int p = 0; p < P; ++p) {
         tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;
@@ -150,7 +162,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     const int T = cfg.prefix_tiles_per_item > 0
                       ? cfg.prefix_tiles_per_item
                       : choose_prefix_tiles_per_item(tiles, groups, rows_per_split, rows_per_item > kPrefixTileRows ? 1.6 : 1.0,
-                                                     cfg.head_dim, cfg.num_sms);
+                                                     cfg.head_dim, cfg.num_sms, any_suffix ? 0.35 : 0.0);
     plan->prefix_tiles_per_item = T;
 
     plan->sample_info.assign(size_t(B), SampleInfo{});

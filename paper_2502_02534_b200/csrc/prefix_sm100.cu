@@ -242,7 +242,8 @@ template <int D, bool kTwo, bool kLowReg>
 __device__ __forceinline__ void
 prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensorMap *pmap_v,
             const PrefixItem *__restrict__ items, int group, int causal, float scale_log2,
-            float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+            float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status, int *launch_counter,
+            int *done_counter)
 {
     constexpr int kKeys = prefix_tile_keys<kLowReg>();   // keys per tile
     using L = PrefixSmem<D, kTwo, kKeys>;
@@ -273,6 +274,11 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kAbortOff);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // A counted launch (fused step) announces itself to the merge stage.  This may happen before the wait for the
+    // preceding grid: if that grid is the previous step's merge stage, all of its warps have read the counters by
+    // the time they let this grid start.  Doing it here hides the round trip behind the set-up.
+    if (launch_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0)
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(launch_counter) : "memory");
     const int4 it0 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));
     const int4 it1 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x) + 1);
     const int first_token = it0.x, n_keys = it0.y, kv = it0.z, first_sample = it0.w;
@@ -306,6 +312,9 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     // while that kernel drained; from here on it reads inputs and (later) overwrites partial results, so the
     // predecessor must be complete.  Only then may our own dependent (the suffix stage) start beside us.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the announcement of a counted launch (see the top of the kernel) is visible before this block lets the suffix
+    // grid -- and with it the merge grid -- start
+    if (launch_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0) __threadfence();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kProducerWarp) {
@@ -623,6 +632,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         }
         __syncthreads();
     }
+    // Every result of this block is stored (the barrier above): count the block off for the merge stage of a fused
+    // step, which is ordered behind the suffix grid only.
+    if (done_counter != nullptr && threadIdx.x == 0)   // a release reduction: nothing comes back, the thread does not wait
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(done_counter) : "memory");
     if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem_base, L::kTmemCols);
@@ -633,9 +646,11 @@ template <int D>
 __global__ void __launch_bounds__(320, 1)
 prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
-                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status,
+                   int *launch_counter, int *done_counter)
 {
-    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, true, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status, launch_counter,
+                           done_counter);
 }
 
 // At most 144 registers per thread: two of these warps and one suffix warp (208) fit the 512 registers per lane of
@@ -644,9 +659,11 @@ template <int D>
 __global__ void __maxnreg__(144)
 prefix_kernel_one(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
-                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+                  float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status,
+                   int *launch_counter, int *done_counter)
 {
-    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, true>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status, launch_counter,
+                           done_counter);
 }
 
 // One row tile, long items: the block owns the SM anyway (long ring), so S stays in registers.
@@ -654,9 +671,11 @@ template <int D>
 __global__ void __launch_bounds__(224, 1)
 prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
-                       float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status)
+                       float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status,
+                        int *launch_counter, int *done_counter)
 {
-    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status);
+    prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status, launch_counter,
+                            done_counter);
 }
 
 // Self-test of the bounded wait: one block waits on a barrier that nothing ever arrives on.  The wait must give
@@ -742,7 +761,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     lc.attrs = &attr;
     lc.numAttrs = 1;   // set-up may overlap the tail of the preceding kernel; the kernel waits before touching memory
     return int(cudaLaunchKernelEx(&lc, kern, mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, int(a.causal), scale_log2, a.partial_o,
-                                  a.partial_lse, a.status));
+                                  a.partial_lse, a.status, a.launch_counter, a.done_counter));
 }
 
 }  // namespace

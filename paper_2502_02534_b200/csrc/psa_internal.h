@@ -17,6 +17,13 @@ constexpr int kPrefixTileKeys = 128;   // keys per tensor-core tile (N of QK^T, 
 constexpr int kPrefixTileRows = 128;   // query rows per softmax warpgroup (M of one MMA)
 constexpr int kPrefixRowsPerItem = 256;// two row tiles share the K/V stream of one thread block
 constexpr int kStatusWords = 64;       // int32 words reserved at the start of the workspace
+// Words of that area besides word 0 (the status).  Within one fused step the suffix grid runs beside the prefix grid
+// and the merge grid is ordered behind the SUFFIX grid only, so the prefix grid announces itself and counts its
+// blocks off here, and merge warps wait (bounded) until the count reaches launches x blocks.  Neither word is ever
+// reset by a kernel (both wrap around together); binding a workspace zeroes them.
+constexpr int kPrefixLaunchWord = 8;   // counted prefix launches so far (block 0 adds 1 before it releases the suffix grid)
+static_assert(kPrefixLaunchWord % 2 == 0, "the two counters are read as one aligned 64-bit word");
+constexpr int kPrefixDoneWord = kPrefixLaunchWord + 1;     // prefix blocks of all those launches that have stored their partial results
 
 // One thread block of the prefix stage: a (prompt, kv head, row group, key range).
 struct PrefixItem {
@@ -143,6 +150,8 @@ struct PrefixArgs {
     bool causal = false;  // prefill: row (token) i sees keys up to its own packed token index
     float *partial_o, *partial_lse;  // device
     int32_t *status;                 // device
+    int32_t *launch_counter = nullptr, *done_counter = nullptr;   // device; when set: block 0 adds 1 to the first at its start,
+                                                                  // every block adds 1 to the second after storing its results
 };
 int launch_prefix(const PrefixArgs &a, void *stream, std::string *err);
 int launch_bounded_wait_selftest(int32_t *status, unsigned long long limit_ns, void *stream);
@@ -170,6 +179,11 @@ struct MergeArgs {
     void *out;
     float *lse;
     bool after_stage = false;  // launched right behind a prefix / suffix stage of the same step
+    // fused step with both stages: wait until *prefix_done reaches *prefix_launches x prefix_blocks before reading
+    // prefix partials
+    const int32_t *prefix_counters = nullptr;   // the pair (kPrefixLaunchWord, kPrefixDoneWord), read as one 64-bit word
+    int32_t *status = nullptr;
+    int32_t prefix_blocks = 0;
 };
 int launch_merge(const MergeArgs &a, void *stream, std::string *err);
 

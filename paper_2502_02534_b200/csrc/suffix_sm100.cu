@@ -101,10 +101,7 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     int S = __ldg(suffix_lens + s);
     S = min(S, __ldg(&sample_info[s].suf_len_bound));
     const int n_tok = min(S - tok0, chunk_tokens);
-    if (n_tok <= 0) {  // the merge stage derives the chunk count from the same length
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        return;
-    }
+    if (n_tok <= 0) return;  // the merge stage derives the chunk count from the same length
     const int n_pages = (n_tok + kPageSize - 1) / kPageSize;
     const int my_pages = (n_pages - warp + kWarps - 1) / kWarps;  // pages warp, warp+4, ...
     const int32_t *my_page_ids = page_indices + __ldg(page_indptr + s) + tok0 / kPageSize;
@@ -257,11 +254,11 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
         partial_o[size_t(prow0 + g) * D + d] = acc / z;
         if (d == 0) partial_lse[prow0 + g] = (top + log2f(z)) * 0.6931471805599453f;
     }
-    // When launched as a programmatic dependent of the prefix stage this grid runs beside it.  The merge
-    // stage may be scheduled once every block is here, and no block retires before the prefix grid has
-    // completed, so that "suffix grid complete" implies "prefix grid complete" for the merge stage.
+    // When launched as a programmatic dependent of the prefix stage this grid runs beside it, and its blocks retire
+    // as soon as they are done (so that the next ones take their place while prefix blocks still run): the merge
+    // stage, ordered behind this grid, learns of the prefix grid's completion through a counter.  It may be
+    // scheduled once every block is here.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 template <int D, int G>
