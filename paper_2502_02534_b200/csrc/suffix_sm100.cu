@@ -122,11 +122,25 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     const __nv_bfloat16 *head_k = pool_k + int64_t(kv) * stride_head;
     const __nv_bfloat16 *head_v = pool_v + int64_t(kv) * stride_head;
 
-    // copy page number i of this warp (tokens [16*(warp+4i), +16) of the chunk) into ring slot i % kStages
+    // Page ids of this warp's pages, 32 at a time: lane l holds the id of page number 32 g + l of the warp, for the
+    // group g in use (ids_cur) and the next one (ids_nxt).  One coalesced load per group instead of one dependent
+    // load per page: otherwise every copy would wait a full L2 round trip for its address first.
+    auto load_ids = [&](int g) {
+        const int i = g * 32 + lane;
+        return i < my_pages ? __ldg(my_page_ids + warp + i * kWarps) : 0;
+    };
+    int ids_cur = load_ids(0), ids_nxt = load_ids(1);
+
+    // copy page number i of this warp (tokens [16*(warp+4i), +16) of the chunk) into ring slot i % kStages;
+    // called with i = 0, 1, 2, ... in order
     auto issue_page = [&](int i) {
+        if (i > 0 && (i & 31) == 0) {   // warp-uniform: the next group of ids becomes the current one
+            ids_cur = ids_nxt;
+            ids_nxt = load_ids((i >> 5) + 1);
+        }
+        const int64_t page = __shfl_sync(0xffffffffu, ids_cur, i & 31);
         if (i < my_pages) {
             const int page_in_chunk = warp + i * kWarps;
-            const int64_t page = __ldg(my_page_ids + page_in_chunk);
             const int valid = min(kPageSize, n_tok - page_in_chunk * kPageSize);
             const uint32_t dst = warp_smem + (i % kStages) * L::kStageBytes;
             const __nv_bfloat16 *src_k = head_k + page * stride_page;
