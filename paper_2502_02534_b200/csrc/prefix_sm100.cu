@@ -296,7 +296,9 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         *abort_flag = 0;
         mbar_init(bar_q(), 1);
         for (int i = 0; i < kMaxRing; ++i) { mbar_init(bar_full(i), 1); mbar_init(bar_empty(i), 1); }
-        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128); }
+        // p[t]: one arrival per softmax thread of row tile t; with two row tiles p[0] also takes the arrival of the
+        // thread that watches the K/V tiles land (see the MMA issuers)
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128 + ((kTwo && t == 0) ? 1 : 0)); }
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
@@ -368,7 +370,19 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             auto next_slot = [&](int sl, int by) { sl += by; return sl >= ring ? sl - ring : sl; };
             if constexpr (kTwo) {
                 // Two row tiles: ONE issuer, which alternates between the tiles (two threads issuing into the same
-                // pipe measured slower here: 95 us instead of 77 us on 2048 rows x 8192 keys x 8 heads).
+                // pipe measured slower here: 95 us instead of 77 us on 2048 rows x 8192 keys x 8 heads).  The second
+                // thread only watches the K/V tiles land: per key tile j it waits for V_j and K_{j+1} and then adds
+                // its arrival to p[0], so that the issuer, whose every poll costs the tensor pipe idle time, has one
+                // wait per row tile and key tile (P ready, which now also says "operands landed") instead of three.
+                if (who == 1) {
+                    bool landed = true;
+                    for (int j = 0; landed && j < n_tiles; ++j) {
+                        if (j > 0) landed = mbar_wait(bar_p(0), sphase(j - 1), abort_flag);   // one arrival per phase of p[0]
+                        if (landed) landed = wait_entry(2 * j + 1);                           // V_j
+                        if (landed && j + 1 < n_tiles) landed = wait_entry(2 * j + 2);        // K_{j+1}
+                        if (landed) mbar_arrive(bar_p(0));
+                    }
+                }
                 bool ok = who == 0;
                 if (ok) ok = mbar_wait(bar_q(), 0, abort_flag);
                 if (ok) ok = wait_entry(0);   // K_0
@@ -380,9 +394,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 int vslot = 1;   // ring slot of V_j; K_{j+1} is in the next one
                 for (int j = 0; ok && j < n_tiles; ++j) {
                     const int kslot = next_slot(vslot, 1);
-                    if (!(ok = wait_entry(2 * j + 1))) break;                       // V_j
-                    if (j + 1 < n_tiles && !(ok = wait_entry(2 * j + 2))) break;    // K_{j+1}
                     for (int t = 0; t < n_rt; ++t) {
+                        // p[0] of tile j completes only after V_j and K_{j+1} have landed (the watcher's arrival)
                         if (!(ok = mbar_wait(bar_p(t), sphase(j), abort_flag))) break;
                         tc_fence_after();
                         issue_pv(t, tmem_base + kColS + t * 128 /* P over S */, vslot, j == 0);
@@ -643,7 +656,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 }
 
 template <int D>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(352, 1)
 prefix_kernel_two(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
                   float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status,
@@ -752,7 +765,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(a.num_items);
-    lc.blockDim = dim3(kTwo ? 320 : 224);   // softmax warps, producer, one (two row tiles) or two MMA issuers
+    lc.blockDim = dim3(kTwo ? 352 : 224);   // softmax warps, producer, two more single-thread warps (MMA issuers / watcher)
     lc.dynamicSmemBytes = L::total(ring);
     lc.stream = st;
     cudaLaunchAttribute attr{};
