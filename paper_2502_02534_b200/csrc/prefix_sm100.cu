@@ -14,20 +14,24 @@
 // query row.  Per key tile and row tile:  S = Q K^T (SS MMA, K-major operands, 128-byte swizzle) -> the softmax
 // warpgroup reads S from TMEM and writes P (bf16) back to TMEM -> O += P V (TS MMA, P from TMEM, V as MN-major B
 // operand).  K/V are read from HBM/L2 once per item.  Three shapes of block, chosen per launch from the plan:
-//   two row tiles (some item has > 128 rows), 10 warps, 128-key tiles, ring of 5 tiles:
+//   two row tiles (some item has > 128 rows), 11 warps, 128-key tiles, ring of 5 tiles:
 //     warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1
 //     warp 8           TMA producer: Q once, then K and V tiles through a ring of buffers
 //     warp 9           MMA issuer (one lane) and owner of the TMEM allocation
+//     warp 10          watcher (one lane): waits for the K/V tiles of each key tile to land and adds its arrival to
+//                      the P barrier of row tile 0, so that the issuer polls one barrier per row tile and key tile
 //     The two row tiles alternate on the tensor pipe (one tile's softmax overlaps the other's MMAs); P is written
 //     over S.  TMEM: S0 S1 at columns 0 / 128, O0 O1 at 256 / 256 + D.
-//   one row tile, small (<= 128 rows; short items, or enough rows not to be purely HBM-bound), 7 warps
-//     (0-3 softmax, 4 producer, 5 issuer of QK^T, 6 issuer of PV: the issuing thread polls barriers and commits
-//     between batches of MMAs, a few hundred cycles of scalar code per tile during which the tensor pipe drains, so
-//     two issuers whose waits overlap each other's MMAs shorten the key-tile period), <= 144 registers, 129 KB of shared memory: ONE SUFFIX BLOCK FITS BESIDE IT
+//   one row tile, small (<= 128 rows; short items, or enough rows not to be purely HBM-bound), 8 warps:
+//     0-3 softmax, 4 producer, 5 issuer of QK^T, 6 issuer of PV, 7 watcher.  The issuing thread is a serial
+//     bottleneck -- between two batches of MMAs it polls barriers and commits, a few hundred cycles of scalar code
+//     per tile during which the tensor pipe drains -- so the two kinds of MMA have an issuer each, whose waits
+//     overlap the other's MMAs.  <= 144 registers, 129 KB of shared memory: ONE SUFFIX BLOCK FITS BESIDE IT
 //     on the SM.  64-key tiles through a ring of 6 (three tiles of look-ahead in 96 KB); S0/S1 alternate by key
 //     tile so that QK^T of tile j+1 runs under the softmax of tile j; P has TMEM columns of its own (384..511),
 //     which keeps S intact and makes the common softmax a single pass against the current reference maximum.
-//   one row tile, long (<= 64 rows and long items: HBM-bound): the same with 128-key tiles and a ring of 6; owns the SM.
+//   one row tile, long (<= 64 rows and long items: HBM-bound): the same with 128-key tiles, a ring of 6 and no
+//     watcher (7 warps); owns the SM.
 // The epilogue sends O / l through a padded staging tile laid over the idle ring, so that every global store
 // instruction writes one full row.  Launched as a programmatic dependent: set-up (barriers, TMEM) overlaps the
 // tail of the preceding kernel, `griddepcontrol.wait` precedes the first memory access, and the suffix stage is
@@ -206,8 +210,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
            (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
 }
 
-// Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 10 warps); otherwise one row
-// tile (one Q tile, 7 warps).
+// Shared-memory plan of one block.  kTwo: two row tiles (two Q tiles, 11 warps); otherwise one row
+// tile (one Q tile, 7 or 8 warps).
 constexpr int kMaxRing = 6;
 // Ring length per block shape: 5 x 32 KB beside two Q tiles, else 6 (never fewer buffers than the epilogue
 // staging tile needs).
@@ -250,6 +254,12 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     constexpr int ring = prefix_ring<D, kTwo, kLowReg>();   // K/V tile buffers in flight
     constexpr int kSoftmaxWarps = kTwo ? 8 : 4;
     constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1, kMmaWarp2 = kSoftmaxWarps + 2;
+    constexpr int kWatchWarp = kSoftmaxWarps + 3;   // one row tile only (with two row tiles the second issuer warp watches)
+    // A watcher thread folds the "K/V tile landed" waits into the P barriers.  Measured: it pays in the two-row-tile
+    // block (69 instead of 78 us on 2048 rows x 8192 keys x 8 heads) and in the small block that shares its SM with
+    // a suffix block (whole step 59.1 instead of 61.6 us on 64 samples x 16384 + U[0,2048] tokens, although that
+    // block alone gets 4 % slower); the long one-row-tile block is 4 % slower with it and goes without.
+    constexpr bool kWatch = kTwo || kLowReg;
     constexpr int kKSteps = D / 16;                 // MMA k-steps of QK^T
     constexpr int kPSteps = kKeys / 16;   // MMA k-steps of PV
     constexpr uint32_t kIdescQK = make_idesc(kKeys, false);
@@ -297,8 +307,9 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         mbar_init(bar_q(), 1);
         for (int i = 0; i < kMaxRing; ++i) { mbar_init(bar_full(i), 1); mbar_init(bar_empty(i), 1); }
         // p[t]: one arrival per softmax thread of row tile t; with two row tiles p[0] also takes the arrival of the
-        // thread that watches the K/V tiles land (see the MMA issuers)
-        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128 + ((kTwo && t == 0) ? 1 : 0)); }
+        // thread that watches the K/V tiles land (see the MMA issuers); with one row tile both p[] are per key tile
+        // and both take it
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128 + ((kWatch && (!kTwo || t == 0)) ? 1 : 0)); }
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
@@ -421,7 +432,8 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 }
                 int kslot = 4 % ring;   // ring slot of K_{j+2} = entry 2j+4
                 for (int j = 0; ok && j + 2 < n_tiles; ++j) {
-                    if (!(ok = wait_entry(2 * j + 4))) break;
+                    // p[j & 1] of tile j: P handed over and, with a watcher, V_j and K_{j+2} landed (its arrival)
+                    if (!kWatch && !(ok = wait_entry(2 * j + 4))) break;
                     if (!(ok = mbar_wait(bar_p(j & 1), sphase(j), abort_flag))) break;
                     tc_fence_after();
                     issue_qk(0, j & 1, kslot);
@@ -434,13 +446,25 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 bool ok = true;
                 int vslot = 1 % ring;   // ring slot of V_j = entry 2j+1
                 for (int j = 0; ok && j < n_tiles; ++j) {
-                    if (!(ok = wait_entry(2 * j + 1))) break;
+                    if (!kWatch && !(ok = wait_entry(2 * j + 1))) break;
                     if (!(ok = mbar_wait(bar_p(j & 1), sphase(j), abort_flag))) break;
                     tc_fence_after();
                     issue_pv(0, tmem_base + kColP + (j & 1) * 64, vslot, j == 0);
                     tc_commit(bar_empty(vslot));
                     vslot = next_slot(vslot, 2);
                 }
+            }
+        }
+    } else if (!kTwo && kWatch && warp == kWatchWarp) {
+        // ------------------------------------------------------------ watcher (one row tile): per key tile j it waits
+        // for V_j and K_{j+2} to land and then adds its arrival to p[j & 1], so that the two issuers poll one barrier each
+        if (lane == 0) {
+            bool landed = true;
+            for (int j = 0; landed && j < n_tiles; ++j) {
+                if (j >= 2) landed = mbar_wait(bar_p(j & 1), sphase(j - 2), abort_flag);   // one arrival per phase
+                if (landed) landed = mbar_wait(bar_full((2 * j + 1) % ring), ((2 * j + 1) / ring) & 1, abort_flag);
+                if (landed && j + 2 < n_tiles) landed = mbar_wait(bar_full((2 * j + 4) % ring), ((2 * j + 4) / ring) & 1, abort_flag);
+                if (landed) mbar_arrive(bar_p(j & 1));
             }
         }
     } else if (warp < 4 * n_rt) {
@@ -765,7 +789,7 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
     const float scale_log2 = a.sm_scale * 1.4426950408889634f;
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(a.num_items);
-    lc.blockDim = dim3(kTwo ? 352 : 224);   // softmax warps, producer, two more single-thread warps (MMA issuers / watcher)
+    lc.blockDim = dim3(kTwo ? 352 : (kShape == 1 ? 256 : 224));   // softmax warps, producer, two more single-thread warps (MMA issuers / watcher)
     lc.dynamicSmemBytes = L::total(ring);
     lc.stream = st;
     cudaLaunchAttribute attr{};
