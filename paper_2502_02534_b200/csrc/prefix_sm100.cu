@@ -513,38 +513,63 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 
             float ps[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial row sums
             if constexpr (kTwo) {
-                // ---- S in registers; P (bf16) is written back over the first 64 columns of S
+                // ---- S in registers; P (bf16) is written back over the first 64 columns of S.
+                // Common case: ONE pass that exponentiates against the current reference maximum while tracking the
+                // largest exponent.  Only if that exceeds the threshold (or on a row's first visible keys) is S read
+                // again from tensor memory -- P has not been stored yet, so it is still there -- and the tile redone
+                // the classic way: maximum, move the reference (rescaling O), exponentials.
+                auto load_s = [&]() {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
-                tmem_wait_ld();
-                float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (valid < kKeys) {   // last tile of a ragged prompt: masked keys become -inf
+                    for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sreg[c]);
+                    tmem_wait_ld();
+                    if (valid < kKeys) {   // last tile of a ragged prompt, or the diagonal of a prefill: masked keys become -inf
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;
+                    }
+                };
+                auto exp_in_place = [&](float &xmax) {   // sreg: 128 scores -> 64 words of packed bf16 P (in sreg[0], sreg[1])
+                    const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // a row that has seen no key yet: exponentiate against 0
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            const float x0 = fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_use);
+                            const float x1 = fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_use);
+                            mx[(i >> 1) & 3] = fmaxf(mx[(i >> 1) & 3], fmaxf(x0, x1));
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                            ps[(i >> 1) & 3] += p0 + p1;
+                            sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                        }
+                    }
+                    xmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                };
+                load_s();
+                bool redo = j == 0;   // nothing to exponentiate against yet
+                if (j > 0) {
+                    float xmax;
+                    exp_in_place(xmax);
+                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold || (m_ref == -INFINITY && xmax != -INFINITY));
+                    if (redo) load_s();
+                }
+                if (redo) {
+                    float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(sreg[c][i]));   // eight independent chains
-                const float tmax = scale_log2 * fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                // move the reference maximum only when a logit exceeds it by more than the threshold
-                const bool need = tmax > m_ref + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, need)) {
-                    if (!(ok = move_reference(need, tmax))) break;
-                }
-                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // a row that has seen no key yet: p = 2^(-inf) = 0
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_use));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_use));
-                        ps[(i >> 1) & 3] += p0 + p1;
-                        sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                        for (int i = 0; i < 32; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(sreg[c][i]));   // eight independent chains
+                    const float tmax = scale_log2 * fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                    // move the reference maximum only when a logit exceeds it by more than the threshold
+                    const bool need = tmax > m_ref + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        if (!(ok = move_reference(need, tmax))) break;
                     }
+                    float xmax;
+                    exp_in_place(xmax);
                 }
                 tmem_st32(s_addr, sreg[0]);
                 tmem_st32(s_addr + 32, sreg[1]);
