@@ -170,7 +170,10 @@ int32_t psa_plan_suffix_items(const psa_plan_t *plan, int32_t *items4);
  *   out            [B, Hq, D] device, bf16 or f32 per cfg.out_dtype.
  *   lse            [B, Hq] f32 device, natural logarithm; -inf for an empty context (out = 0).
  *   workspace      the buffer bound with psa_plan_bind_workspace.
- * Concurrent calls must use distinct workspaces.
+ * The prefix and suffix stages run side by side; the merge stage, which stream order puts behind the suffix
+ * stage only, learns that the prefix stage is complete from two counters kept in the workspace's status area
+ * (bounded wait; PSA_ERR_TIMEOUT in the status word if it ever ran out).  The counters belong to the workspace:
+ * calls that share one must be ordered on one stream, concurrent calls must use distinct workspaces.
  */
 psa_status_t psa_decode(const psa_plan_t *plan, const void *q,
                         const void *prefix_k, const void *prefix_v, const int64_t prefix_strides[2],

@@ -22,14 +22,21 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // group of `tiles` tiles is cut into ceil(tiles / T) items.  Items are dispatched longest first to the SMs, so
 // the stage takes about max(longest item, sum of items / SMs); every split also costs a partial result per row
 // (4*D bytes written, read again by the merge stage).  Costs are in tile steps of a one-row-tile block (~1.5 us);
-// a step of a two-row-tile block counts 1.6.  In a step that also has a suffix stage the two grids run side by side
+// a step of a two-row-tile block counts 1.3.  In a step that also has a suffix stage the two grids run side by side
 // and the suffix stage (HBM-bound, the longer one) wants every SM, so the SM time the prefix items take is charged
 // once more at `sm_time_weight` (measured on 32 samples x 4096 + U[0,1024] tokens: 88 items of 3 tiles give a 22.2 us
 // step, 128 items of 2 tiles 23.4 us, although the prefix stage alone is faster with 128).  Pick the T with the
 // smallest estimate, larger T on ties.
+//
+// Blocks of two row tiles own their SM (no suffix block fits beside them) and work in the tensor-bound regime, where
+// they need little of the HBM bandwidth.  There the whole step is estimated instead: while the prefix items run,
+// the suffix stage streams on the SMs they leave free, at up to 72 GB/s per SM (measured: 84 free SMs sustain
+// 6.1 TB/s) and at most what the prefix stage leaves of 6.4 TB/s; afterwards it has the machine to itself.  Few long
+// items then beat many short ones: 2048 rows x 8192 keys x 8 heads beside 2.1 GB of suffix K/V take 338 us as 64
+// items of 64 tiles against 385 us as 128 items of 32 tiles.
 int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::vector<int64_t> &groups,
                                  const std::vector<int64_t> &partial_rows_per_split, double step_weight, int head_dim, int num_sms,
-                                 double sm_time_weight)
+                                 double sm_time_weight, bool owns_sm, double prefix_bytes, double suffix_bytes)
 {
     int64_t max_tiles = 0;
     for (int64_t t : tiles) max_tiles = std::max(max_tiles, t);
@@ -39,16 +46,26 @@ int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::v
     double best_cost = std::numeric_limits<double>::infinity();
     int best_T = 1;
     for (int64_t T = 1; T <= max_tiles; ++T) {
-        double sum = 0.0, longest = 0.0, partial = 0.0;
+        double sum = 0.0, longest = 0.0, partial = 0.0, items = 0.0;
         for (size_t p = 0; p < tiles.size(); ++p) {
             if (tiles[p] == 0) continue;
             const int64_t splits = ceil_div(tiles[p], T);
             const double len = step_weight * double(ceil_div(tiles[p], splits)) + overhead;
             sum += double(groups[p] * splits) * len;
+            items += double(groups[p] * splits);
             longest = std::max(longest, len);
             partial += double(partial_rows_per_split[p] * splits) * steps_per_partial_row;
         }
-        const double cost = std::max(longest, 1.1 * sum / num_sms) + partial + sm_time_weight * sum / num_sms;
+        double cost = std::max(longest, 1.1 * sum / num_sms) + partial;
+        if (owns_sm && suffix_bytes > 0.0) {
+            const double step_us = 1.5, hbm = 6.4e6 /* bytes per us */, per_sm = 7.2e4;
+            const double t_prefix = std::max(longest, 1.1 * sum / num_sms) * step_us;
+            const double free_sms = std::max(0.0, double(num_sms) - items);
+            const double rate = std::max(0.0, std::min(hbm - prefix_bytes / t_prefix, free_sms * per_sm));
+            cost += std::max(0.0, suffix_bytes - rate * t_prefix) / hbm / step_us;
+        } else {
+            cost += sm_time_weight * sum / num_sms;
+        }
         if (cost <= best_cost) { best_cost = cost; best_T = int(T); }
     }
     return best_T;
@@ -152,7 +169,13 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
                                                            : (max_rows >= 2 * kPrefixRowsPerItem ? kPrefixRowsPerItem : kPrefixTileRows);
     const int samples_per_group = rows_per_item / G;
     bool any_suffix = false;
-    for (int64_t s = 0; s < B; ++s) any_suffix = any_suffix || suffix_lens[s] > 0;
+    double suffix_kv_bytes = 0.0, prefix_kv_bytes = 0.0;   // K and V, bf16, all heads
+    for (int64_t s = 0; s < B; ++s) {
+        any_suffix = any_suffix || suffix_lens[s] > 0;
+        suffix_kv_bytes += 4.0 * double(suffix_lens[s]) * cfg.num_kv_heads * cfg.head_dim;
+    }
+    for (int p = 0; p < P; ++p)
+        if (n_samples[p] > 0) prefix_kv_bytes += 4.0 * double(prefix_lens[p]) * cfg.num_kv_heads * cfg.head_dim;
     std::vector<int64_t> tiles(P), groups(P), rows_per_split(P);
     for (int p = 0; p < P; ++p) {
         tiles[p] = n_samples[p] > 0 ? ceil_div(prefix_lens[p], kPrefixTileKeys) : 0;
@@ -161,8 +184,9 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
     }
     const int T = cfg.prefix_tiles_per_item > 0
                       ? cfg.prefix_tiles_per_item
-                      : choose_prefix_tiles_per_item(tiles, groups, rows_per_split, rows_per_item > kPrefixTileRows ? 1.6 : 1.0,
-                                                     cfg.head_dim, cfg.num_sms, any_suffix ? 0.35 : 0.0);
+                      : choose_prefix_tiles_per_item(tiles, groups, rows_per_split, rows_per_item > kPrefixTileRows ? 1.3 : 1.0,
+                                                     cfg.head_dim, cfg.num_sms, any_suffix ? 0.35 : 0.0,
+                                                     rows_per_item > kPrefixTileRows, prefix_kv_bytes, suffix_kv_bytes);
     plan->prefix_tiles_per_item = T;
 
     plan->sample_info.assign(size_t(B), SampleInfo{});

@@ -81,8 +81,9 @@ def test_planner_fills_the_machine_on_the_named_configurations():
             continue
         L, N, S = wl.draw_lengths(cfg)
         info = make_plan(L, N, S, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim).info
-        # the two stages run side by side: the prefix stage takes at least half of the SMs, the rest is left to the suffix stage
-        assert info.num_prefix_items >= 0.5 * 148, name
+        # the two stages run side by side: the prefix stage takes a good part of the SMs (fewer, longer items when it is
+        # tensor-bound and the suffix stage can use the bandwidth meanwhile), the rest is left to the suffix stage
+        assert info.num_prefix_items >= 0.4 * 148, name
         # the suffix stage is bound by HBM as a whole: at least one block per SM, and enough of them in flight
         assert info.num_suffix_items >= 1.5 * 148, name
 
