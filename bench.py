@@ -30,8 +30,8 @@ UNIT = "sample-tokens/s"
 L2_BYTES = 126e6
 # DRAM bytes (read + write) per launch of the dominant kernel, from an ncu launch list of this very command
 # (dram__bytes_read.sum + dram__bytes_write.sum).  Only valid for the kernel source it was taken with.
-NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68270655 + 16007,
-                        "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "93c285341b3d3d1f"}}
+NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68270729 + 12211,
+                        "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "2792110b60f06e29"}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -301,6 +301,15 @@ def run_psa(args, cfg):
             t_roof_ms = max(abytes[name] / (hbm * 1e9), aflops[name] / (tf * 1e12)) * 1e3
             kernels[name] = {"ms": stage_avg[name], "algorithmic_bytes": abytes[name], "flops": aflops[name],
                              "t_roof_ms": t_roof_ms, "frac_of_roofline": t_roof_ms / stage_avg[name] if stage_avg[name] else None}
+        # The planner may run a tensor-bound prefix stage on part of the SMs on purpose (few long items, so that the
+        # suffix stage streams beside it); the tensor fraction on the SMs the stage actually occupies says how well
+        # each of them is used.
+        n_sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        blocks = info.num_prefix_items
+        if stage_avg["prefix"] and blocks:
+            share = min(1.0, blocks / n_sms)
+            kernels["prefix"].update({"blocks": blocks, "sms": n_sms,
+                                      "tensor_frac_on_sms_used": aflops["prefix"] / (tf * 1e12 * share) / (stage_avg["prefix"] * 1e-3)})
         kernels["merge"] = {"ms": stage_avg["merge"]}
         t_roof_step = max((abytes["prefix"] + abytes["suffix"]) / (hbm * 1e9), (aflops["prefix"] + aflops["suffix"]) / (tf * 1e12)) * 1e3
         # CPU baseline: the oracle as it stands, on this machine's host cores, one full step of the same workload
