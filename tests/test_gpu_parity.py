@@ -232,6 +232,68 @@ def test_stage_entry_points_compose_to_decode():
     assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, "stages")
 
 
+def test_many_fused_steps_on_one_workspace_and_counter_wrap_around():
+    """The merge stage of a fused step learns that the prefix stage is complete from two counters in the workspace
+    (prefix launches, prefix blocks done) that no kernel ever resets.  Many steps in a row, a stand-alone prefix stage
+    in between (it must not count), a CUDA-graph replay, and counters preset just below 2^32 so that they wrap
+    during the run: every step must give the oracle's result."""
+    import torch
+    from paper_2502_02534_b200 import decode
+    w = wl.make_workload(cfg(prefix_len=(900, 900), suffix_len=(0, 300), samples_per_prefix=40), poison=True)
+    ref_o, ref_l, _ = oracle.attend(w)
+    dev = to_device(w)
+    plan = make_plan(w, "f32", num_sms=16)      # few SMs in the plan: several prefix blocks per SM, several waves
+    plan.bind_workspace()
+    n_blocks = plan.info.num_prefix_items
+    assert n_blocks > 1 and plan.info.num_suffix_items > 0
+    B, Hq, D = int(np.sum(w["n_samples"])), w["num_q_heads"], w["head_dim"]
+    out = torch.empty((B, Hq, D), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+
+    def step(stage="all"):
+        decode(plan, dev["q"], dev["prefix_k"], dev["prefix_v"], dev["pool_k"], dev["pool_v"], dev["page_indptr"],
+               dev["page_indices"], dev["suffix_lens"], out, lse, stage=stage)
+
+    def check(what):
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, what)
+
+    for i in range(25):
+        out.fill_(float("nan")); lse.fill_(float("nan"))
+        step()
+        if i % 6 == 0:
+            check(f"step {i}")
+        if i % 5 == 0:
+            step("prefix")                      # a stand-alone stage leaves the counters alone
+    check("after 25 steps")
+    words = plan.workspace[:64 * 4].view(torch.int32)
+    assert int(words[8]) == 25 and int(words[9]) == 25 * n_blocks
+
+    # preset the counters a few launches below the wrap of the 32-bit product launches x blocks
+    launches = (2 ** 32 - 3 * n_blocks) // n_blocks
+    words[8] = int(np.array(launches, dtype=np.uint32).view(np.int32)) if launches >= 2 ** 31 else launches
+    words[9] = int(np.array((launches * n_blocks) % 2 ** 32, dtype=np.uint32).view(np.int32))
+    torch.cuda.synchronize()
+    for i in range(8):
+        out.fill_(float("nan")); lse.fill_(float("nan"))
+        step()
+        check(f"wrap step {i}")
+
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            step()
+        side.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(6):
+                step()
+    out.fill_(float("nan"))
+    g.replay(); g.replay()
+    check("graph replays")
+
+
 def test_decode_from_host_buffers():
     import torch
     from paper_2502_02534_b200 import decode_host
