@@ -275,6 +275,30 @@ psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * The step after the path, second half: draw the next token of every sample from its logits.  The paper samples its
+ * candidate answers at temperature T in {0.4, 0.7, 1.0} with a seed (appendix "Experiment details").  Row r gets
+ *     tokens[r] = argmax_i ( logits[r, i] / T_r + g_i ),   g_i = -ln(-ln u_i)          (ties: lowest i)
+ * (the Gumbel-max identity: token i comes out with probability softmax(logits[r] / T_r)_i); T_r = 0 means greedy
+ * decoding, argmax_i logits[r, i].  The uniforms are Philox4x32-10 words (Salmon et al., SC'11): counter
+ * (i / 4, step, r, 0), key (low, high word of seeds[r]), u_i = ((word[i % 4] >> 9) + 0.5) * 2^-23, so a draw depends
+ * only on (seeds[r], step, r, i): pass the decode step as `step` and keep the seeds fixed to get reproducible runs.
+ *
+ *   logits        [num_rows, vocab] device, bf16 (PSA_OUT_BF16) or f32 (PSA_OUT_F32) per `logits_dtype`, 16-byte
+ *                 aligned, element (r, i) at r*row_stride + i; row_stride >= vocab, a multiple of 8 elements.
+ *   temperature   [num_rows] f32 device (<= 0 or NaN: greedy);  seeds [num_rows] u64 device.
+ *   tokens        [num_rows] int32 device, out.
+ *   scratch       device, 8-byte aligned, psa_sample_scratch_bytes(num_rows) bytes; caller-owned, cleared and
+ *                 overwritten by every call (calls that share it must be ordered on one stream).
+ * Arithmetic is fp32 (scores are compared in fp32).  Only enqueues work (a memset and two kernels) on `cuda_stream`.
+ * num_rows <= 65535.  -inf logits are never drawn unless the whole row is -inf (then token 0); NaN logits are
+ * not supported.
+ */
+size_t psa_sample_scratch_bytes(int32_t num_rows);
+psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
+                               const float *temperature, const uint64_t *seeds, uint32_t step, int32_t *tokens,
+                               void *scratch, size_t scratch_bytes, void *cuda_stream);
+
+/*
  * Self-test of the device-side error path (no counterpart in the paper).  Enqueues one tiny kernel whose only
  * wait is on a barrier that nothing completes; the wait gives up after `limit_ns` (<= 1 s), the kernel writes
  * PSA_ERR_TIMEOUT into the status word of `workspace` and exits normally.  psa_check_status then reports and

@@ -8,7 +8,7 @@ Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 
 published definition, so that a (seed, step, row, vocabulary index) names one number on every machine:
 
     counter = (index // 4, step, row, 0),  key = (seed low word, seed high word),
-    u = ((x >> 8) + 0.5) * 2^-24  for the word x = output[index % 4].
+    u = ((x >> 9) + 0.5) * 2^-23  for the word x = output[index % 4].   (23 bits: what an fp32 mantissa holds exactly)
 
 Everything after the generator is fp64.  Ties go to the lowest index.
 """
@@ -45,7 +45,7 @@ def uniforms(seed: int, step: int, row: int, vocab: int) -> np.ndarray:
     words = philox4x32_10((blk, z + np.uint32(step & 0xFFFFFFFF), z + np.uint32(row & 0xFFFFFFFF), z),
                           (np.uint32(seed & 0xFFFFFFFF), np.uint32((seed >> 32) & 0xFFFFFFFF)))
     x = np.choose((idx % np.uint64(4)).astype(np.int64), [words[0], words[1], words[2], words[3]])
-    return ((x >> np.uint32(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+    return ((x >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
 def scores(logits_row: np.ndarray, temperature: float, seed: int, step: int, row: int) -> np.ndarray:

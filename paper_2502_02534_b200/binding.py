@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_create_prefill", "psa_prefill", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -106,6 +106,10 @@ def library():
         lib.psa_append_kv.argtypes = [P, P, P, P, P, POINTER(c_int64), P, P, P, P, c_size_t, P]
         lib.psa_validate_page_table.restype = c_int32
         lib.psa_validate_page_table.argtypes = [P, P, P, P, c_int64, P, c_size_t, P]
+        lib.psa_sample_scratch_bytes.restype = c_size_t
+        lib.psa_sample_scratch_bytes.argtypes = [c_int32]
+        lib.psa_sample_tokens.restype = c_int32
+        lib.psa_sample_tokens.argtypes = [P, c_int32, c_int64, c_int32, c_int32, P, P, ctypes.c_uint32, P, P, c_size_t, P]
         lib.psa_selftest_bounded_wait.restype = c_int32
         lib.psa_selftest_bounded_wait.argtypes = [P, c_size_t, ctypes.c_uint64, P]
         lib.psa_status_string.restype = c_char_p
@@ -303,6 +307,25 @@ def append_kv(plan: Plan, new_k, new_v, suffix_k_pool, suffix_v_pool, page_indpt
     _check(library().psa_append_kv(plan.handle, _ptr(new_k), _ptr(new_v), _ptr(suffix_k_pool), _ptr(suffix_v_pool), qst,
                                    _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens), _ptr(plan.workspace),
                                    plan.workspace.numel(), _stream_ptr(stream)))
+
+
+def sample_tokens(logits, temperature, seeds, step, tokens=None, scratch=None, *, stream=None):
+    """psa_sample_tokens on torch CUDA tensors: logits [B, V] (bf16 or f32, rows may be padded: stride(0) >= V),
+    temperature [B] f32, seeds [B] int64 (bit pattern of the u64 seed).  Returns the int32 token tensor."""
+    import torch
+    lib = library()
+    B, V = logits.shape
+    dtype = {torch.bfloat16: PSA_OUT_BF16, torch.float32: PSA_OUT_F32}[logits.dtype]
+    if logits.stride(1) != 1:
+        raise ValueError("logits must be contiguous along the vocabulary")
+    if tokens is None:
+        tokens = torch.empty(B, dtype=torch.int32, device=logits.device)
+    need = int(lib.psa_sample_scratch_bytes(B))
+    if scratch is None:
+        scratch = torch.empty(max(8, need), dtype=torch.uint8, device=logits.device)
+    _check(lib.psa_sample_tokens(_ptr(logits), dtype, logits.stride(0), B, V, _ptr(temperature), _ptr(seeds), int(step) & 0xFFFFFFFF,
+                                 _ptr(tokens), _ptr(scratch), scratch.numel(), _stream_ptr(stream)))
+    return tokens
 
 
 def decode_host(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,
