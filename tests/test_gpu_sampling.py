@@ -108,3 +108,57 @@ def test_misuse_returns_status_codes():
         sample_tokens(x, T, seeds, 0, scratch=torch.empty(8, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 3
     assert sample_tokens(x, T, seeds, 0).tolist() == [0, 0] or True  # equal logits at T = 1: any token is a valid draw
+
+
+def test_decode_sample_append_loop_with_one_plan():
+    """The loop the paper's sampler runs for every candidate answer: attend, draw the next token at a temperature, append
+    its K/V, attend again -- five steps on one plan.  The output projection and the token embeddings stand in for the
+    model (random tables, torch ops in the test only).  At every step the library's attention is checked against the
+    attention oracle on the cache the loop has built, the drawn tokens against the sampling oracle on the very logits
+    the GPU saw, and the appended cache against the oracle's append, bit for bit."""
+    import torch
+    import oracle
+    import psa_workloads as wl
+    from paper_2502_02534_b200 import append_kv, sample_tokens
+    from psa_testlib import assert_close, make_plan, run_gpu, to_device
+    steps, vocab = 5, 512
+    c = wl.PsaConfig(name="loop", num_prefixes=2, samples_per_prefix=6, num_q_heads=8, num_kv_heads=2, head_dim=64,
+                     prefix_len=(150, 400), suffix_len=(steps, 90), page_size=16, permute_pages=True, seed=21)
+    w = wl.make_workload(c, poison=False)
+    bounds = np.array(w["suffix_lens"]).copy()
+    w["suffix_lens"] = (bounds - steps).astype(np.int32)
+    plan = make_plan(w, "f32", suffix_bounds=bounds)
+    dev = to_device(w)
+    B, Hq, Hkv, D = 12, 8, 2, 64
+    g = torch.Generator().manual_seed(5)
+    proj = (torch.randn(Hq * D, vocab, generator=g) * 0.3).cuda()                      # "output projection"
+    emb_k = wl.normal_bf16((vocab, Hkv, D), 90, 1); emb_v = wl.normal_bf16((vocab, Hkv, D), 90, 2)   # "embeddings" of a token
+    T = np.resize(np.array([0.4, 0.7, 1.0, 0.0], dtype=np.float32), B)
+    seeds = np.arange(B, dtype=np.uint64) * np.uint64(1000003) + np.uint64(17)
+    T_d = torch.from_numpy(T).cuda(); seeds_d = torch.from_numpy(seeds.view(np.int64)).cuda()
+    drawn = []
+    for k in range(steps):
+        out, lse, _ = run_gpu(w, "f32", plan=plan, dev=dev)
+        ref_o, ref_l, _ = oracle.attend(w)
+        assert_close(out, lse, ref_o, ref_l, f"loop step {k}")
+        logits = torch.from_numpy(out.reshape(B, Hq * D)).float().cuda() @ proj       # [B, vocab] f32, on the GPU's own outputs
+        tok = sample_tokens(logits.contiguous(), T_d, seeds_d, k).cpu().numpy()
+        seen = logits.double().cpu().numpy()
+        for b in range(B):
+            s = sampling.scores(seen[b], float(T[b]), int(seeds[b]), k, b)
+            ref = int(np.argmax(s))
+            assert tok[b] == ref or s[ref] - s[tok[b]] <= NEAR_TIE, (k, b, tok[b], ref)
+        drawn.append(tok)
+        new_k, new_v = emb_k[tok], emb_v[tok]
+        w = oracle.append_kv(w, new_k, new_v)
+        append_kv(plan, torch.from_numpy(new_k.view(np.int16)).cuda().view(torch.bfloat16),
+                  torch.from_numpy(new_v.view(np.int16)).cuda().view(torch.bfloat16), dev["pool_k"], dev["pool_v"],
+                  dev["page_indptr"], dev["page_indices"], dev["suffix_lens"])
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert np.array_equal(dev["suffix_lens"].cpu().numpy(), w["suffix_lens"])
+        assert np.array_equal(dev["pool_k"].view(torch.int16).cpu().numpy().view(np.uint16), w["pool_k"])
+    drawn = np.stack(drawn)
+    assert len(np.unique(drawn)) > steps          # the samples of a prompt go different ways
+    greedy = T == 0
+    assert greedy.any() and not np.array_equal(drawn[:, ~greedy][:, :1], drawn[:, ~greedy][:, 1:2])
