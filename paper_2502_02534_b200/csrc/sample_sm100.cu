@@ -20,6 +20,7 @@
 
 #include <algorithm>
 #include <string>
+#include <type_traits>
 
 #include "psa_internal.h"
 
@@ -84,36 +85,51 @@ sample_kernel(const void *__restrict__ logits, int64_t row_stride, int vocab, in
     const int g0 = split * per, g1 = min(n_groups, g0 + per);
     float best = -INFINITY;
     uint32_t best_i = 0xFFFFFFFFu;   // "nothing seen": loses against every real index at equal score
-    for (int g = g0 + threadIdx.x; g < g1; g += kSampleThreads) {
-        const int i0 = g * 4;
-        float x[4];
-        if (i0 + 3 < vocab) {
-            if constexpr (kF32) {
-                const float4 v = __ldcs(reinterpret_cast<const float4 *>(static_cast<const float *>(logits) + row * row_stride + i0));
-                x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-            } else {
-                const uint2 v = __ldcs(reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(logits) + row * row_stride + i0));
-                x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
-                x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
-            }
-        } else {   // the ragged last group of the row
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                x[e] = -INFINITY;
-                if (i0 + e < vocab) {
-                    if constexpr (kF32) x[e] = static_cast<const float *>(logits)[row * row_stride + i0 + e];
-                    else x[e] = __bfloat162float(static_cast<const __nv_bfloat16 *>(logits)[row * row_stride + i0 + e]);
-                }
-            }
-        }
+    // scores of the four logits x[] of group g (indices 4g .. 4g+3, the first `valid` of them inside the row)
+    auto consume = [&](int g, const float (&x)[4], int valid) {
         uint32_t r[4] = {0u, 0u, 0u, 0u};
         if (!greedy) philox4x32_10(uint32_t(g), step, uint32_t(row), 0u, k0, k1, r);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float s = x[e];
             if (!greedy) s = fmaf(x[e], inv_t, gumbel(r[e] >> 9));
-            if (i0 + e < vocab && (s > best || best_i == 0xFFFFFFFFu)) { best = s; best_i = uint32_t(i0 + e); }   // first maximum wins
+            if (e < valid && (s > best || best_i == 0xFFFFFFFFu)) { best = s; best_i = uint32_t(4 * g + e); }   // first maximum wins
         }
+    };
+    // full groups: one vector load each, the next one in flight while this one is worked on
+    using Vec = typename std::conditional<kF32, float4, uint2>::type;
+    const Vec *base = reinterpret_cast<const Vec *>(kF32 ? static_cast<const void *>(static_cast<const float *>(logits) + row * row_stride)
+                                                         : static_cast<const void *>(static_cast<const __nv_bfloat16 *>(logits) + row * row_stride));
+    const int full_end = min(g1, vocab / 4);
+    int g = g0 + threadIdx.x;
+    Vec cur{};
+    if (g < full_end) cur = __ldcs(base + g);
+    for (; g < full_end; g += kSampleThreads) {
+        Vec nxt{};
+        if (g + kSampleThreads < full_end) nxt = __ldcs(base + g + kSampleThreads);
+        float x[4];
+        if constexpr (kF32) {
+            x[0] = cur.x; x[1] = cur.y; x[2] = cur.z; x[3] = cur.w;
+        } else {
+            x[0] = __uint_as_float(cur.x << 16); x[1] = __uint_as_float(cur.x & 0xFFFF0000u);
+            x[2] = __uint_as_float(cur.y << 16); x[3] = __uint_as_float(cur.y & 0xFFFF0000u);
+        }
+        consume(g, x, 4);
+        cur = nxt;
+    }
+    // the ragged last group of the row (vocab not a multiple of 4): one thread of the block that owns it
+    const int tail = vocab / 4;
+    if ((vocab & 3) && tail >= g0 && tail < g1 && threadIdx.x == 0) {
+        float x[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            x[e] = -INFINITY;
+            if (4 * tail + e < vocab) {
+                if constexpr (kF32) x[e] = static_cast<const float *>(logits)[row * row_stride + 4 * tail + e];
+                else x[e] = __bfloat162float(static_cast<const __nv_bfloat16 *>(logits)[row * row_stride + 4 * tail + e]);
+            }
+        }
+        consume(tail, x, vocab & 3);
     }
     unsigned long long key = best_i == 0xFFFFFFFFu ? 0ull : make_key(best, best_i);
 #pragma unroll
