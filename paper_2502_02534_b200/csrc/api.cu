@@ -1,5 +1,6 @@
 // C ABI of the library (include/psa.h): argument checks, workspace carving, stage launches.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cstring>
@@ -23,6 +24,14 @@ psa_status_t cuda_fail(cudaError_t e, const char *what)
     return fail(PSA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
 }
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// A named range on the host timeline of profilers (NVTX; a pointer check when no tool is attached).
+struct TraceRange {
+    explicit TraceRange(const char *name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+    TraceRange(const TraceRange &) = delete;
+    TraceRange &operator=(const TraceRange &) = delete;
+};
 
 struct Carved {
     int32_t *status;
@@ -197,6 +206,7 @@ static psa_status_t prefix_impl(const psa_plan_t *plan, const void *q, const voi
                                 const int64_t prefix_strides[2], void *workspace, size_t workspace_bytes, void *cuda_stream,
                                 bool count_blocks)
 {
+    TraceRange trace("psa prefix stage");
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
     if (st != PSA_OK) return st;
@@ -235,6 +245,7 @@ static psa_status_t suffix_impl(const psa_plan_t *plan, const void *q, const voi
                                 const int32_t *suffix_lens, void *workspace, size_t workspace_bytes, void *cuda_stream,
                                 bool after_prefix)
 {
+    TraceRange trace("psa suffix stage");
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
     if (st != PSA_OK) return st;
@@ -271,6 +282,7 @@ psa_status_t psa_decode_suffix(const psa_plan_t *plan, const void *q, const void
 static psa_status_t merge_impl(const psa_plan_t *plan, const int32_t *suffix_lens, void *out, float *lse, void *workspace,
                                size_t workspace_bytes, void *cuda_stream, bool after_stage, bool wait_for_prefix_count = false)
 {
+    TraceRange trace("psa merge stage");
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
     if (st != PSA_OK) return st;
@@ -321,6 +333,7 @@ psa_status_t psa_decode(const psa_plan_t *plan, const void *q, const void *prefi
                         void *cuda_stream)
 {
     if (!plan) return fail(PSA_ERR_INVALID_ARG, "null plan");
+    TraceRange trace("psa_decode");
     // The suffix stage is independent of the prefix stage: launched as its programmatic dependent it runs
     // beside it.  The merge stage needs both, but stream order (and the programmatic dependency) only puts it
     // behind the suffix grid, so with both stages present the prefix blocks count themselves off in the workspace
