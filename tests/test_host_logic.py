@@ -88,6 +88,22 @@ def test_planner_fills_the_machine_on_the_named_configurations():
         assert info.num_suffix_items >= 1.5 * 148, name
 
 
+def test_planner_weighs_the_two_stages_against_each_other():
+    """A tensor-bound prefix stage (many rows per KV head) beside a large suffix stage is cut into few long items that
+    leave SMs to the suffix stage; without a suffix stage the same prefix is spread over the whole machine.  Suffix items
+    stay whole samples as long as the longest one is a small part of the stage."""
+    L, N = [8192], [256]
+    big = make_plan(L, N, [2048] * 256, Hq=64, Hkv=8).info
+    none = make_plan(L, N, [0] * 256, Hq=64, Hkv=8).info
+    assert big.num_prefix_items <= 74 < 148 * 0.8 <= none.num_prefix_items
+    assert big.prefix_tiles_per_item > none.prefix_tiles_per_item
+    assert big.suffix_chunk_tokens >= 2048 and big.num_suffix_items == 256 * 8
+    # one very long sample among short ones is still split, so that it does not become the tail of the stage
+    lens = [64] * 63 + [60000]
+    skew = make_plan([128], [64], lens, Hq=32, Hkv=8).info
+    assert skew.suffix_chunk_tokens < 60000 and skew.num_suffix_items > 64 * 8
+
+
 def test_bad_arguments_give_status_codes():
     from paper_2502_02534_b200 import PsaError
     ok = dict(prefix_lens=[10], n_samples=[2], suffix_lens=[1, 2])
