@@ -87,7 +87,7 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
               const int32_t *__restrict__ page_indptr, const int32_t *__restrict__ page_indices,
               const int32_t *__restrict__ suffix_lens, const SuffixItem *__restrict__ items,
               const SampleInfo *__restrict__ sample_info, int num_q_heads, int chunk_tokens, float scale_log2,
-              float *__restrict__ partial_o, float *__restrict__ partial_lse)
+              float *__restrict__ partial_o, float *__restrict__ partial_lse, int first_of_step)
 {
     using L = SuffixSmem<D>;
     constexpr int KK = D / 16;           // k-steps of QK^T
@@ -96,8 +96,16 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     extern __shared__ __align__(128) unsigned char smem_raw[];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int4 item = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));
+    const int4 item = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));   // plan data, bound long before
     const int s = item.x, kv = item.y, tok0 = item.z, prow0 = item.w;
+    // Not behind a prefix stage: this grid is launched as a programmatic dependent of whatever precedes it in the
+    // stream, its blocks got here while that kernel drained, and they wait for it before they touch anything it may
+    // have written (lengths, page table, K/V, Q) or still be reading (partial results).  The next kernel may then
+    // set itself up under this grid.  Behind a prefix stage there is nothing to wait for: the prefix blocks have.
+    if (first_of_step) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
     int S = __ldg(suffix_lens + s);
     S = min(S, __ldg(&sample_info[s].suf_len_bound));
     const int n_tok = min(S - tok0, chunk_tokens);
@@ -272,7 +280,7 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     // as soon as they are done (so that the next ones take their place while prefix blocks still run): the merge
     // stage, ordered behind this grid, learns of the prefix grid's completion through a counter.  It may be
     // scheduled once every block is here.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!first_of_step) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 template <int D, int G>
@@ -298,11 +306,11 @@ int launch_one(const SuffixArgs &a, cudaStream_t st)
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = &attr;
-    lc.numAttrs = a.after_prefix ? 1 : 0;   // run beside the prefix stage launched just before
+    lc.numAttrs = 1;   // behind a prefix stage: runs beside it; else: set-up under the tail of the preceding kernel
     return int(cudaLaunchKernelEx(&lc, kern, static_cast<const __nv_bfloat16 *>(a.q), static_cast<const __nv_bfloat16 *>(a.pool_k),
                                   static_cast<const __nv_bfloat16 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok,
                                   a.page_indptr, a.page_indices, a.suffix_lens, a.items, a.sample_info, a.num_q_heads,
-                                  a.chunk_tokens, scale_log2, a.partial_o, a.partial_lse));
+                                  a.chunk_tokens, scale_log2, a.partial_o, a.partial_lse, a.after_prefix ? 0 : 1));
 }
 
 }  // namespace
