@@ -299,6 +299,21 @@ psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dtype, int64_t
                                void *scratch, size_t scratch_bytes, void *cuda_stream);
 
 /*
+ * The paper's three "attn" tasks (appendix "Benchmark details"): softmax(S) V folded over a stream of keys in the
+ * three forms the paper asks its agents to implement -- task 0 "MaxSum" (running maximum and sum, output normalised at
+ * every step), task 1 "ExpMaxDiff" feeding "DivSum" (maximum split from the sum, still normalised every step), task 2
+ * "ExpMaxDiff" feeding two weighted sums divided once at the end (the form the fast kernels above use).  Plain
+ * CUDA-core reference kernels (one warp per row, one key at a time, fp32), for small problems: they tie the library to
+ * the paper's operator forms, they are not a fast path.
+ *   q [num_rows, head_dim], k, v [num_keys, head_dim]: bf16 device, contiguous; scores are sm_scale * q.k_j.
+ *   out [num_rows, head_dim] f32, m_out, l_out [num_rows] f32: the output and the final running maximum and sum
+ *   (natural exponent; lse = m + ln l).  No keys: out = 0, m = -inf, l = 0, the paper's initial state.
+ * head_dim a multiple of 32, at most 256.  Only enqueues one kernel on `cuda_stream`.
+ */
+psa_status_t psa_attn_task(int32_t task, const void *q, const void *k, const void *v, int32_t num_rows, int32_t num_keys,
+                           int32_t head_dim, float sm_scale, float *out, float *m_out, float *l_out, void *cuda_stream);
+
+/*
  * Self-test of the device-side error path (no counterpart in the paper).  Enqueues one tiny kernel whose only
  * wait is on a barrier that nothing completes; the wait gives up after `limit_ns` (<= 1 s), the kernel writes
  * PSA_ERR_TIMEOUT into the status word of `workspace` and exits normally.  psa_check_status then reports and

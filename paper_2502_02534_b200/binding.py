@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_create_prefill", "psa_prefill", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens", "psa_attn_task",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -110,6 +110,8 @@ def library():
         lib.psa_sample_scratch_bytes.argtypes = [c_int32]
         lib.psa_sample_tokens.restype = c_int32
         lib.psa_sample_tokens.argtypes = [P, c_int32, c_int64, c_int32, c_int32, P, P, ctypes.c_uint32, P, P, c_size_t, P]
+        lib.psa_attn_task.restype = c_int32
+        lib.psa_attn_task.argtypes = [c_int32, P, P, P, c_int32, c_int32, c_int32, c_float, P, P, P, P]
         lib.psa_selftest_bounded_wait.restype = c_int32
         lib.psa_selftest_bounded_wait.argtypes = [P, c_size_t, ctypes.c_uint64, P]
         lib.psa_status_string.restype = c_char_p
@@ -326,6 +328,19 @@ def sample_tokens(logits, temperature, seeds, step, tokens=None, scratch=None, *
     _check(lib.psa_sample_tokens(_ptr(logits), dtype, logits.stride(0), B, V, _ptr(temperature), _ptr(seeds), int(step) & 0xFFFFFFFF,
                                  _ptr(tokens), _ptr(scratch), scratch.numel(), _stream_ptr(stream)))
     return tokens
+
+
+def attn_task(task, q, k, v, sm_scale, *, stream=None):
+    """psa_attn_task on torch CUDA tensors: q [R, D], k / v [M, D] bf16.  Returns (out [R, D] f32, m [R], l [R])."""
+    import torch
+    R, D = q.shape
+    M = k.shape[0]
+    out = torch.empty((R, D), dtype=torch.float32, device=q.device)
+    m = torch.empty(R, dtype=torch.float32, device=q.device)
+    l = torch.empty(R, dtype=torch.float32, device=q.device)
+    _check(library().psa_attn_task(int(task), _ptr(q), _ptr(k) if M else None, _ptr(v) if M else None, R, M, D, float(sm_scale),
+                                   _ptr(out), _ptr(m), _ptr(l), _stream_ptr(stream)))
+    return out, m, l
 
 
 def decode_host(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,

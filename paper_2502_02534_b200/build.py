@@ -11,7 +11,7 @@ HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libpsa.so"
-SOURCES = ["api.cu", "plan.cpp", "prefix_sm100.cu", "suffix_sm100.cu", "merge_sm100.cu", "static_workspace.cu", "append_sm100.cu", "sample_sm100.cu"]
+SOURCES = ["api.cu", "plan.cpp", "prefix_sm100.cu", "suffix_sm100.cu", "merge_sm100.cu", "static_workspace.cu", "append_sm100.cu", "sample_sm100.cu", "attn_tasks.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v", f"-I{INCLUDE}", f"-I{CSRC}",
