@@ -79,6 +79,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
                 asm volatile("ld.acquire.gpu.global.b64 %0, [%1];" : "=l"(both) : "l"(prefix_counters) : "memory");
                 lag = int(uint32_t(both) * uint32_t(prefix_blocks) - uint32_t(both >> 32));
                 if (lag <= 0) break;
+                __nanosleep(200);   // the prefix stage may still run for a while (long prompts, short suffixes): poll gently
                 if ((spins & 255u) == 255u) {
                     unsigned long long now;
                     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));

@@ -490,3 +490,18 @@ def test_page_table_validator_flags_bad_tables_only():
     expect_bad(dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], pool=1)
     plan.validate_page_table(dev["page_indptr"], dev["page_indices"], dev["suffix_lens"], n_pool)
     plan.check_status()
+
+
+def test_long_prefix_beside_tiny_suffixes_merge_waits_for_the_prefix_stage():
+    """The suffix stage is over long before the prefix stage here, so the merge grid really has to wait on the prefix
+    block counter (and, planned lengths aside, some samples have no suffix token at all at run time)."""
+    import torch
+    from paper_2502_02534_b200 import decode
+    w = wl.make_workload(cfg(prefix_len=(6000, 6000), suffix_len=(1, 3), samples_per_prefix=40, num_q_heads=16, num_kv_heads=2),
+                         poison=True)
+    plan = make_plan(w, "f32", prefix_tiles_per_item=47, suffix_bounds=np.asarray(w["suffix_lens"]) + 4)   # few long prefix items
+    w["suffix_lens"] = np.asarray(w["suffix_lens"]).copy(); w["suffix_lens"][::3] = 0
+    ref_o, ref_l, _ = oracle.attend(w)
+    for _ in range(3):
+        out, lse, _ = run_gpu(w, "f32", plan=plan)
+        assert_close(out, lse, ref_o, ref_l, "long prefix, tiny suffixes")
