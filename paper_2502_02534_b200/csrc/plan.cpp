@@ -78,14 +78,16 @@ int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::v
 //     max( (sum of tokens + 384 per item) / min(slots, items),  longest item / 3 + 384 ).
 // The 384 is what a block spends finding its pages (three dependent loads) and combining its warps, expressed
 // in tokens.  Measured on B200: 64 samples x U[0,2048] tokens take 41.9 us as whole-sample items (0.98 of the
-// copy bandwidth), 45.4 us in 1024-token chunks, 48.7 us in 512-token chunks.
+// copy bandwidth), 45.4 us in 1024-token chunks, 48.7 us in 512-token chunks; 32 samples x U[0,1024] tokens beside a
+// 4096-token prefix: the step takes 21.3 us with 896-token chunks, 21.7 with 768, 22.1 with 1024, 22.8 with 512.
 int choose_suffix_chunk(const int32_t *lens, int n, int num_kv_heads, int num_sms)
 {
     const double overhead = 384.0;
     const double slots = 2.0 * num_sms;
     double best_cost = std::numeric_limits<double>::infinity();
     int best = 64;
-    for (int C = 64; C <= 8192; C *= 2) {
+    // candidates: every 64 tokens up to 1024, every 256 up to 4096, every 1024 up to 8192
+    for (int C = 64; C <= 8192; C += (C < 1024 ? 64 : (C < 4096 ? 256 : 1024))) {
         double sum = 0.0, items = 0.0;
         int64_t longest = 0;
         for (int s = 0; s < n; ++s) {
