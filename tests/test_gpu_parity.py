@@ -505,3 +505,30 @@ def test_long_prefix_beside_tiny_suffixes_merge_waits_for_the_prefix_stage():
     for _ in range(3):
         out, lse, _ = run_gpu(w, "f32", plan=plan)
         assert_close(out, lse, ref_o, ref_l, "long prefix, tiny suffixes")
+
+
+def test_two_plans_on_two_streams_with_their_own_workspaces():
+    """Concurrent steps are allowed on distinct workspaces: two different problems, each on its own stream, interleaved
+    call by call, several rounds without a synchronisation in between."""
+    import torch
+    from paper_2502_02534_b200 import decode
+    probs = []
+    for seed, n, L in ((31, 24, 1800), (32, 40, 700)):
+        w = wl.make_workload(cfg(prefix_len=(L, L), suffix_len=(0, 500), samples_per_prefix=n, seed=seed), poison=True)
+        plan = make_plan(w, "f32"); plan.bind_workspace()
+        dev = to_device(w)
+        B, Hq, D = n, w["num_q_heads"], w["head_dim"]
+        out = torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
+        lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+        probs.append((w, plan, dev, out, lse, torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for _ in range(6):
+        for w, plan, dev, out, lse, st in probs:
+            decode(plan, dev["q"], dev["prefix_k"], dev["prefix_v"], dev["pool_k"], dev["pool_v"], dev["page_indptr"],
+                   dev["page_indices"], dev["suffix_lens"], out, lse, stream=st)
+    torch.cuda.synchronize()
+    for w, plan, dev, out, lse, st in probs:
+        plan.check_status()
+        ref_o, ref_l, _ = oracle.attend(w)
+        B, Hq, D = out.shape
+        assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, "two streams")
