@@ -354,7 +354,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         // A single issuing thread is a serial bottleneck: between two batches of MMAs it polls barriers and commits,
         // a few hundred cycles of scalar code each time, during which the tensor pipe drains and idles.  With two
         // issuers the waits of one overlap the MMAs of the other.
-        //   two row tiles: issuer 0 alone (see there)
+        //   two row tiles: thread 0 issues everything, thread 1 only watches the K/V tiles land (see there)
         //   one row tile:  issuer 0 issues every QK^T, issuer 1 every PV
         if (lane == 0) {
             const int who = warp - kMmaWarp;
