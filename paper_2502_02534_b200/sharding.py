@@ -1,7 +1,12 @@
-"""Multi-GPU plumbing: the path shards over independent prompts, with no data-path collective.
+"""Multi-GPU plumbing.  Nothing here computes attention.
 
-Each rank owns a contiguous range of prompts (with all of their samples), plans and decodes it
-alone, and only timing / result bookkeeping crosses ranks.  Nothing here computes attention.
+Two ways to cut the path, both without any communication inside the attention itself:
+  * by prompt (`partition_prompts`, `shard_workload`): each rank owns a contiguous range of prompts with all of their
+    samples, plans and decodes it alone; no data-path collective at all, only timing crosses ranks.
+  * by KV head (`shard_heads`, `gather_heads`): each rank holds the prefix K/V and the suffix pools of its KV heads
+    and the matching query heads of every sample, runs the whole step on `[B, Hq / world, D]`, and ONE exchange
+    follows: an all-gather of the outputs along the head axis (B * Hq * D elements in total).  This keeps the
+    shared prefix shared on every rank; sharding by sample would replicate its read.
 """
 from __future__ import annotations
 
@@ -51,6 +56,44 @@ def shard_workload(w: dict, rank: int, world: int) -> dict:
         sample_range=(s0, s1),
     )
     return sub
+
+
+def shard_heads(w: dict, rank: int, world: int) -> dict:
+    """The sub-problem of one rank under KV-head sharding: KV heads [rank * Hkv / world, (rank + 1) * Hkv / world) and
+    their query heads, for every sample.  Lengths, page table and sample order are unchanged."""
+    Hq, Hkv = int(w["num_q_heads"]), int(w["num_kv_heads"])
+    if Hkv % world:
+        raise ValueError(f"{Hkv} KV heads do not divide over {world} ranks")
+    hk = Hkv // world
+    G = Hq // Hkv
+    k0, k1 = rank * hk, (rank + 1) * hk
+    sub = dict(w)
+    sub.update(
+        num_q_heads=hk * G, num_kv_heads=hk,
+        q=np.ascontiguousarray(np.asarray(w["q"])[:, k0 * G:k1 * G]),
+        prefix_k=np.ascontiguousarray(np.asarray(w["prefix_k"])[:, k0:k1]),
+        prefix_v=np.ascontiguousarray(np.asarray(w["prefix_v"])[:, k0:k1]),
+        pool_k=np.ascontiguousarray(np.asarray(w["pool_k"])[:, k0:k1]),
+        pool_v=np.ascontiguousarray(np.asarray(w["pool_v"])[:, k0:k1]),
+        head_range=(k0 * G, k1 * G),
+    )
+    return sub
+
+
+def gather_heads(out_local, lse_local):
+    """The one exchange step of KV-head sharding: all-gather of every rank's `out [B, Hq / world, D]` and
+    `lse [B, Hq / world]` (torch tensors, on the device of the process group's backend) along the head axis.
+    Returns (out [B, Hq, D], lse [B, Hq]); without a process group the inputs come back unchanged."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return out_local, lse_local
+    world = dist.get_world_size()
+    outs = [torch.empty_like(out_local) for _ in range(world)]
+    lses = [torch.empty_like(lse_local) for _ in range(world)]
+    dist.all_gather(outs, out_local.contiguous())
+    dist.all_gather(lses, lse_local.contiguous())
+    return torch.cat(outs, dim=1), torch.cat(lses, dim=1)
 
 
 def max_over_ranks(values):

@@ -53,6 +53,45 @@ def test_prompt_sharding_over_two_gloo_ranks(tmp_path):
     assert covered == int(np.sum(w["n_samples"]))
 
 
+def _head_worker(rank, world, port, tmpdir):
+    sys.path.insert(0, ROOT)
+    import torch
+    import torch.distributed as dist
+    import oracle
+    import psa_workloads as wl
+    from paper_2502_02534_b200.sharding import gather_heads, shard_heads
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    cfg = wl.PsaConfig("hs", 2, 5, 8, 4, 16, (30, 90), (0, 50), page_size=16, permute_pages=True, seed=4)
+    w = wl.make_workload(cfg, poison=True)
+    sub = shard_heads(w, rank, world)
+    B, hq, D = 10, sub["num_q_heads"], 16
+    out, lse, _ = oracle.attend(sub, n_threads=1)                       # the oracle stands in for the GPU step of this rank
+    full_o, full_l = gather_heads(torch.from_numpy(out.reshape(B, hq, D)), torch.from_numpy(lse.reshape(B, hq)))
+    np.savez(os.path.join(tmpdir, f"h{rank}.npz"), out=full_o.numpy(), lse=full_l.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_kv_head_sharding_and_its_all_gather_over_two_gloo_ranks(tmp_path):
+    """Each rank attends with half of the KV heads (and their query heads); one all-gather along the head axis gives
+    every rank the unsharded result, bit for bit."""
+    import torch.multiprocessing as mp
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_head_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    sys.path.insert(0, ROOT)
+    import oracle
+    import psa_workloads as wl
+    cfg = wl.PsaConfig("hs", 2, 5, 8, 4, 16, (30, 90), (0, 50), page_size=16, permute_pages=True, seed=4)
+    w = wl.make_workload(cfg, poison=True)
+    ref_o, ref_l, _ = oracle.attend(w)
+    for r in range(2):
+        z = np.load(tmp_path / f"h{r}.npz")
+        assert np.array_equal(z["out"].reshape(-1, 16), ref_o) and np.array_equal(z["lse"].reshape(-1), ref_l)
+
+
 def test_partition_is_contiguous_complete_and_balanced():
     from paper_2502_02534_b200.sharding import partition_prompts
     rng = np.random.default_rng(0)
