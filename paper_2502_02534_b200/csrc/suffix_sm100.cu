@@ -13,10 +13,14 @@
 //     4 KB contiguous (D = 128), so every copy instruction of a warp reads 512
 //     consecutive bytes.  No block-wide barrier in the main loop.
 //   * the dot products run on warp-level tensor-core MMAs (m16n8k16, bf16 in, fp32
-//     accumulate) with the G query rows padded to 16: plain FMAs could not keep up
-//     with HBM at G = 8.  K fragments come from ldmatrix, V fragments from
-//     ldmatrix.trans, both conflict-free through a 16-byte XOR swizzle of the rows.
-//   * row maxima are refreshed lazily: the quad shuffle + rescale only runs when some
+//     accumulate), computed TRANSPOSED so that the G (<= 8) query rows are the MMA's
+//     8-wide side and nothing is padded: S^T = K Q^T (16 tokens x 8 rows) and
+//     O^T = V^T P^T (16 channels x 8 rows), one MMA per 16 channels each -- half the
+//     MMAs of the untransposed form, whose 16-row side would be half zeros.  Plain FMAs
+//     could not keep up with HBM at G = 8.  K fragments come from ldmatrix, V^T
+//     fragments from ldmatrix.trans, both conflict-free through a 16-byte XOR swizzle
+//     of the rows; P^T comes from the S^T accumulators through two movmatrix transposes.
+//   * row maxima are refreshed lazily: the shuffles + rescale only run when some
 //     logit exceeds the reference maximum by more than 2^8.
 //   * slots of the last page beyond the sample's length are zero-filled by the copy
 //     (source size 0), never read from memory, and masked to -inf before the softmax.
@@ -59,6 +63,13 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// transpose of an 8x8 matrix of 16-bit elements held in the fragment layout (row = lane / 4, columns 2 * (lane % 4), +1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ float fast_exp2(float x)
 {
     float y;
@@ -91,7 +102,7 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
 {
     using L = SuffixSmem<D>;
     constexpr int KK = D / 16;           // k-steps of QK^T
-    constexpr int DN = D / 8;            // n-tiles of PV
+    constexpr int DT = D / 16;           // 16-channel tiles of O^T
     constexpr int CPR = L::kRowBytes / 16;  // 16-byte chunks per token row
     extern __shared__ __align__(128) unsigned char smem_raw[];
 
@@ -114,15 +125,16 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     const int my_pages = (n_pages - warp + kWarps - 1) / kWarps;  // pages warp, warp+4, ...
     const int32_t *my_page_ids = page_indices + __ldg(page_indptr + s) + tok0 / kPageSize;
 
-    // ---- query fragments: rows g < G of a 16-row tile; rows >= G stay zero
+    // ---- Q^T as the B operand (16 channels x 8 rows per k-step): row lane / 4, channels 2 * (lane % 4), +1 and those
+    // + 8; rows >= G stay zero
     const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    uint32_t qa0[KK], qa2[KK];
+    uint32_t qb0[KK], qb1[KK];
     {
         const __nv_bfloat16 *qp = q + (size_t(s) * num_q_heads + size_t(kv) * G + qrow) * D + qcol;
 #pragma unroll
         for (int kk = 0; kk < KK; ++kk) {
-            qa0[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16)) : 0u;
-            qa2[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16 + 8)) : 0u;
+            qb0[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16)) : 0u;
+            qb1[kk] = qrow < G ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16 + 8)) : 0u;
         }
     }
 
@@ -166,98 +178,116 @@ suffix_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
         cp_async_commit();  // an empty group keeps the group count uniform
     };
 
-    float o[DN][4];
+    // Accumulator layout of the transposed products: a thread holds query rows r0 = 2 * (lane % 4) and r0 + 1, for
+    // tokens (S^T) or channels (O^T) lane / 4 and lane / 4 + 8 of each 16-wide tile: [0], [1] = rows r0, r0 + 1 of the
+    // first, [2], [3] of the second.
+    const int trow = lane >> 2, r0 = (lane & 3) * 2;
+    float o[DT][4];
 #pragma unroll
-    for (int n = 0; n < DN; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-    float m_ref = -INFINITY;  // reference maximum of row qrow, in log2 units (uniform over the quad)
-    float l_part = 0.f;       // this thread's share of the row sum
+    for (int n = 0; n < DT; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+    float m_ref[2] = {-INFINITY, -INFINITY};  // reference maxima of rows r0, r0 + 1, log2 units (same in all 8 lanes that hold the row)
+    float l_part[2] = {0.f, 0.f};             // this thread's share of the two row sums
 
 #pragma unroll
     for (int i = 0; i < kStages - 1; ++i) issue_page(i);
 
     for (int i = 0; i < my_pages; ++i) {
-        cp_async_wait<kStages - 2>();
+        // Refill the slot read in iteration i - 1 BEFORE waiting for page i: while the warp waits, kStages pages are
+        // in flight, not kStages - 1 (the blocks of a small step are bound by the latency of their own copies).
         __syncwarp();
-        issue_page(i + kStages - 1);  // refills the slot read in iteration i - 1
+        issue_page(i + kStages - 1);
+        cp_async_wait<kStages - 1>();
+        __syncwarp();
 
         const int page_in_chunk = warp + i * kWarps;
         const int valid = min(kPageSize, n_tok - page_in_chunk * kPageSize);
         const uint32_t sk = warp_smem + (i % kStages) * L::kStageBytes;
         const uint32_t sv = sk + L::kPageBytes;
 
-        // ---- S = Q K^T for 16 tokens: two 16x8 accumulators
-        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // ---- S^T = K Q^T for 16 tokens x 8 rows; two accumulators halve the dependent chain
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
         {
             const int mat = lane >> 3, r = lane & 7;
-            const int tok = (mat >> 1) * 8 + r;
+            const int tok = (mat & 1) * 8 + r;
             const uint32_t row_addr = sk + tok * L::kRowBytes;
 #pragma unroll
-            for (int kk = 0; kk < KK; ++kk) {
-                const int chunk = 2 * kk + (mat & 1);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4(row_addr + ((chunk ^ (tok & 7)) << 4), b0, b1, b2, b3);
-                mma_bf16(sc[0], qa0[kk], 0u, qa2[kk], 0u, b0, b1);
-                mma_bf16(sc[1], qa0[kk], 0u, qa2[kk], 0u, b2, b3);
+            for (int kk = 0; kk < KK; kk += 2) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4(row_addr + (((2 * kk + (mat >> 1)) ^ (tok & 7)) << 4), a0, a1, a2, a3);
+                mma_bf16(sa, a0, a1, a2, a3, qb0[kk], qb1[kk]);
+                ldmatrix_x4(row_addr + (((2 * kk + 2 + (mat >> 1)) ^ (tok & 7)) << 4), a0, a1, a2, a3);
+                mma_bf16(sb, a0, a1, a2, a3, qb0[kk + 1], qb1[kk + 1]);
             }
         }
-        // this thread holds row qrow, tokens {qcol, qcol+1, 8+qcol, 8+qcol+1}
+        // x[0], x[1]: token trow, rows r0, r0 + 1;  x[2], x[3]: token trow + 8
         float x[4];
-        x[0] = sc[0][0] * scale_log2; x[1] = sc[0][1] * scale_log2;
-        x[2] = sc[1][0] * scale_log2; x[3] = sc[1][1] * scale_log2;
-        if (valid < kPageSize) {
-            if (qcol >= valid) x[0] = -INFINITY;
-            if (qcol + 1 >= valid) x[1] = -INFINITY;
-            if (qcol + 8 >= valid) x[2] = -INFINITY;
-            if (qcol + 9 >= valid) x[3] = -INFINITY;
-        }
-        const float tmax = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-        if (__any_sync(0xffffffffu, tmax > m_ref + kRescaleThreshold)) {
-            float rmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-            rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 2));
-            const float m_new = fmaxf(m_ref, rmax);
-            if (m_new > m_ref) {  // quad-uniform
-                const float alpha = fast_exp2(m_ref - m_new);  // m_ref = -inf gives 0
-                l_part *= alpha;
 #pragma unroll
-                for (int n = 0; n < DN; ++n) { o[n][0] *= alpha; o[n][1] *= alpha; }
-                m_ref = m_new;
+        for (int t = 0; t < 4; ++t) x[t] = (sa[t] + sb[t]) * scale_log2;
+        if (valid < kPageSize) {
+            if (trow >= valid) x[0] = x[1] = -INFINITY;
+            if (trow + 8 >= valid) x[2] = x[3] = -INFINITY;
+        }
+        const float tmax0 = fmaxf(x[0], x[2]), tmax1 = fmaxf(x[1], x[3]);
+        if (__any_sync(0xffffffffu, tmax0 > m_ref[0] + kRescaleThreshold || tmax1 > m_ref[1] + kRescaleThreshold)) {
+            float rmax0 = tmax0, rmax1 = tmax1;   // over the 8 lanes that hold the same rows
+#pragma unroll
+            for (int sh = 4; sh < 32; sh <<= 1) {
+                rmax0 = fmaxf(rmax0, __shfl_xor_sync(0xffffffffu, rmax0, sh));
+                rmax1 = fmaxf(rmax1, __shfl_xor_sync(0xffffffffu, rmax1, sh));
+            }
+            const float m_new0 = fmaxf(m_ref[0], rmax0), m_new1 = fmaxf(m_ref[1], rmax1);
+            if (m_new0 > m_ref[0] || m_new1 > m_ref[1]) {
+                const float alpha0 = m_new0 > m_ref[0] ? fast_exp2(m_ref[0] - m_new0) : 1.f;  // m_ref = -inf gives 0
+                const float alpha1 = m_new1 > m_ref[1] ? fast_exp2(m_ref[1] - m_new1) : 1.f;
+                l_part[0] *= alpha0; l_part[1] *= alpha1;
+#pragma unroll
+                for (int n = 0; n < DT; ++n) { o[n][0] *= alpha0; o[n][1] *= alpha1; o[n][2] *= alpha0; o[n][3] *= alpha1; }
+                m_ref[0] = m_new0; m_ref[1] = m_new1;
             }
         }
         float p[4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) p[t] = fast_exp2(x[t] - m_ref);  // masked slots: exp2(-inf) = 0
-        l_part += (p[0] + p[1]) + (p[2] + p[3]);
-        const uint32_t pa0 = pack_bf16(p[0], p[1]), pa2 = pack_bf16(p[2], p[3]);
+        for (int t = 0; t < 4; ++t) p[t] = fast_exp2(x[t] - m_ref[t & 1]);  // masked slots: exp2(-inf) = 0
+        l_part[0] += p[0] + p[2];
+        l_part[1] += p[1] + p[3];
+        // P^T as the B operand (16 tokens x 8 rows): the two 8x8 halves of S^T's layout, transposed
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p[0], p[1])), pb1 = movmatrix_trans(pack_bf16(p[2], p[3]));
 
-        // ---- O += P V : V[16 tokens x D] read transposed, two 8-wide column tiles per ldmatrix
+        // ---- O^T += V^T P^T : V[16 tokens x D] read transposed, 16 channels per MMA
         {
             const int mat = lane >> 3, r = lane & 7;
-            const int tok = (mat & 1) * 8 + r;
+            const int tok = (mat >> 1) * 8 + r;
             const uint32_t row_addr = sv + tok * L::kRowBytes;
 #pragma unroll
-            for (int n = 0; n < DN; n += 2) {
-                const int chunk = n + (mat >> 1);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(row_addr + ((chunk ^ (tok & 7)) << 4), b0, b1, b2, b3);
-                mma_bf16(o[n], pa0, 0u, pa2, 0u, b0, b1);
-                mma_bf16(o[n + 1], pa0, 0u, pa2, 0u, b2, b3);
+            for (int n = 0; n < DT; ++n) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4_trans(row_addr + (((2 * n + (mat & 1)) ^ (tok & 7)) << 4), a0, a1, a2, a3);
+                mma_bf16(o[n], a0, a1, a2, a3, pb0, pb1);
             }
         }
     }
     cp_async_wait<0>();
 
-    // ---- finish the row sum inside the quad, then combine the 4 warps through shared memory
-    float l_row = l_part + __shfl_xor_sync(0xffffffffu, l_part, 1);
-    l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
+    // ---- finish the row sums over the 8 lanes that share the rows, then combine the 4 warps through shared memory
+    float l_row[2] = {l_part[0], l_part[1]};
+#pragma unroll
+    for (int sh = 4; sh < 32; sh <<= 1) {
+        l_row[0] += __shfl_xor_sync(0xffffffffu, l_row[0], sh);
+        l_row[1] += __shfl_xor_sync(0xffffffffu, l_row[1], sh);
+    }
     __syncthreads();  // every warp is done with its ring: reuse the memory
     float *sm_o = reinterpret_cast<float *>(smem_raw);           // [kWarps][G][D]
     float *sm_m = sm_o + kWarps * G * D;                          // [kWarps][G]
     float *sm_l = sm_m + kWarps * G;                              // [kWarps][G]
-    if (qrow < G) {
-        float *dst = sm_o + (warp * G + qrow) * D + qcol;
 #pragma unroll
-        for (int n = 0; n < DN; ++n) *reinterpret_cast<float2 *>(dst + n * 8) = make_float2(o[n][0], o[n][1]);
-        if ((lane & 3) == 0) { sm_m[warp * G + qrow] = m_ref; sm_l[warp * G + qrow] = l_row; }
+    for (int h = 0; h < 2; ++h) {
+        const int g = r0 + h;
+        if (g < G) {
+            float *dst = sm_o + (warp * G + g) * D + trow;
+#pragma unroll
+            for (int n = 0; n < DT; ++n) { dst[n * 16] = o[n][h]; dst[n * 16 + 8] = o[n][2 + h]; }
+            if (trow == 0) { sm_m[warp * G + g] = m_ref[h]; sm_l[warp * G + g] = l_row[h]; }
+        }
     }
     __syncthreads();
     for (int e = threadIdx.x; e < G * D; e += kWarps * 32) {
