@@ -30,8 +30,8 @@ UNIT = "sample-tokens/s"
 L2_BYTES = 126e6
 # DRAM bytes (read + write) per launch of the dominant kernel, from an ncu launch list of this very command
 # (dram__bytes_read.sum + dram__bytes_write.sum).  Only valid for the kernel source it was taken with.
-NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68271138 + 9926,
-                        "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "5aa1b2d49ef9c8f4"}}
+NCU_TRAFFIC = {"cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68271539 + 18168,
+                        "source": "paper_2502_02534_b200/csrc/suffix_sm100.cu", "sha256_16": "498b791d8050fd97"}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
