@@ -200,11 +200,20 @@ psa_status_t psa_decode(const psa_plan_t *plan, const void *q,
  *     with PSA_ERR_WORKSPACE (the message names both sizes); nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside any stream capture.
+ *   - When the array's memory is taken: the array belongs to a CUDA module of the library, and
+ *     the driver creates it when it loads that module on a device.  Under the runtime's default
+ *     lazy module loading that happens inside the FIRST call on the device -- the one call that
+ *     can still fail for lack of memory, or take milliseconds; with CUDA_MODULE_LOADING=EAGER it
+ *     happens when the library is loaded.  So make one warm-up call per device during
+ *     initialisation, before your own pool claims the remaining memory.  From the second call
+ *     on, free device memory does not change.
  *   - All calls on a device share the one array, and it keeps what the last call left in
  *     it.  Two calls whose GPU work can overlap (different streams, different threads or
  *     different plans) race on it: serialise them, or give one of them psa_decode with its
- *     own workspace.  Device-side status of a step is not retrievable through
- *     psa_check_status here; use psa_decode when that is needed.
+ *     own workspace.
+ *   - Device-side status: every call clears the status word before its kernels run, so read
+ *     it with psa_static_check_status BEFORE the next call if you need it (psa_check_status
+ *     cannot: the array's address is private to the library).
  */
 #define PSA_STATIC_WORKSPACE_BYTES (16u << 20)
 psa_status_t psa_decode_static(const psa_plan_t *plan, const void *q,
@@ -212,6 +221,16 @@ psa_status_t psa_decode_static(const psa_plan_t *plan, const void *q,
                                const void *suffix_k_pool, const void *suffix_v_pool, const int64_t pool_strides[3],
                                const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,
                                void *out, float *lse, void *cuda_stream);
+
+/*
+ * Companions of psa_decode_static (no counterpart in the paper either).  psa_static_check_status synchronises
+ * `cuda_stream`, returns the device-side status word the last psa_decode_static step on the current device left
+ * in the library's array (PSA_OK, PSA_ERR_TIMEOUT or PSA_ERR_BOUNDS) and clears it; it allocates nothing.
+ * psa_static_selftest_bounded_wait is psa_selftest_bounded_wait reporting into that array, so that the error
+ * path can be exercised without a caller workspace.
+ */
+psa_status_t psa_static_check_status(void *cuda_stream);
+psa_status_t psa_static_selftest_bounded_wait(uint64_t limit_ns, void *cuda_stream);
 
 /*
  * The stages one by one, for tests and per-kernel timing.  Same arguments as psa_decode.

@@ -22,11 +22,21 @@ def pass_at_k_enumerated(n, correct, k):
 
 
 def stratify_literal(rates, m):
+    """Section "Stratification and selection", step by step: sort ascending by success rate; lay the sorted list out
+    as m consecutive runs whose sizes differ by at most one, the larger runs first (the reading of "as evenly as
+    possible": the paper does not say where the remainder goes); the success rate of the first element of every run
+    but the first is a boundary value; an experience's level is the number of boundary values it reaches."""
     n = len(rates)
-    order = sorted(range(n), key=lambda i: rates[i])
-    # as even as possible: the first (n % m) runs hold one more ... cut points of the ceil-based even split
-    cuts = [-(-k * n // m) for k in range(1, m)]
-    boundaries = [rates[order[min(c, n - 1)]] for c in cuts]
+    ranked = sorted(rates)
+    runs, pos = [], 0
+    for k in range(m):
+        size = n // m + (1 if k < n % m else 0)
+        runs.append(ranked[pos:pos + size])
+        pos += size
+    boundaries = []
+    for run in runs[1:]:
+        # an empty run (more levels than experiences) starts where the list ends: its boundary is the largest rate
+        boundaries.append(run[0] if run else ranked[-1])
     levels = []
     for r in rates:
         lv = 0

@@ -17,7 +17,7 @@ PSA_OUT_BF16, PSA_OUT_F32 = 0, 1
 EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_create_prefill", "psa_prefill", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
-    "psa_decode", "psa_decode_static", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
+    "psa_decode", "psa_decode_static", "psa_static_check_status", "psa_static_selftest_bounded_wait", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
     "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens", "psa_attn_task",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
@@ -90,6 +90,10 @@ def library():
         lib.psa_decode.argtypes = [P, P, P, P, POINTER(c_int64), P, P, POINTER(c_int64), P, P, P, P, P, P, c_size_t, P]
         lib.psa_decode_static.restype = c_int32
         lib.psa_decode_static.argtypes = [P, P, P, P, POINTER(c_int64), P, P, POINTER(c_int64), P, P, P, P, P, P]
+        lib.psa_static_check_status.restype = c_int32
+        lib.psa_static_check_status.argtypes = [P]
+        lib.psa_static_selftest_bounded_wait.restype = c_int32
+        lib.psa_static_selftest_bounded_wait.argtypes = [ctypes.c_uint64, P]
         lib.psa_decode_prefix.restype = c_int32
         lib.psa_decode_prefix.argtypes = [P, P, P, P, POINTER(c_int64), P, c_size_t, P]
         lib.psa_decode_suffix.restype = c_int32
@@ -289,6 +293,16 @@ def decode_static(plan: Plan, q, prefix_k, prefix_v, suffix_k_pool, suffix_v_poo
     _check(library().psa_decode_static(plan.handle, _ptr(q), _ptr(prefix_k), _ptr(prefix_v), pst, _ptr(suffix_k_pool),
                                        _ptr(suffix_v_pool), qst, _ptr(page_indptr), _ptr(page_indices),
                                        _ptr(suffix_lens), _ptr(out), _ptr(lse), _stream_ptr(stream)))
+
+
+def static_check_status(stream=None):
+    """psa_static_check_status: raise if the last psa_decode_static step left a device-side error; clears it."""
+    _check(library().psa_static_check_status(_stream_ptr(stream)))
+
+
+def static_selftest_bounded_wait(limit_ns=2_000_000, stream=None):
+    """psa_static_selftest_bounded_wait: the unsatisfiable wait, reporting into the library's own array."""
+    _check(library().psa_static_selftest_bounded_wait(int(limit_ns), _stream_ptr(stream)))
 
 
 def prefill(plan: Plan, q, k, v, out, lse, *, kv_strides=None, stream=None):

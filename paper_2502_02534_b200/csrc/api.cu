@@ -434,6 +434,9 @@ psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cud
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "reading the status word");
     if (word != 0) {
+        // The whole status area is cleared, the two prefix counters (launches, blocks done) with it.  That is safe
+        // because the stream is idle here (synchronised above) and the merge stage only compares
+        // launches x blocks with blocks done: both restart from zero together.
         e = cudaMemsetAsync(workspace, 0, sizeof(int32_t) * psa::kStatusWords, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
         if (e != cudaSuccess) return cuda_fail(e, "clearing the status word");

@@ -89,6 +89,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
             }
         }
         lag = __shfl_sync(0xffffffffu, lag, 0);
+        __syncwarp();   // lane 0's acquire load orders the other lanes' reads of the partial results as well
         if (lag > 0) return;   // timed out: the row stays unwritten, the status word says why
     }
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed

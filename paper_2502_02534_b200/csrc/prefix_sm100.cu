@@ -230,7 +230,7 @@ struct PrefixSmem {
     static constexpr int kTileBytes = kHalves * kHalfBytes;           // a K or V tile
     static constexpr int kQTiles = kTwo ? 2 : 1;
     static constexpr int kBarOff = 0;                                 // barriers first, tiles after them
-    static constexpr int kNumBars = 1 + 2 * kMaxRing + 4;             // q, full[], empty[], s_full[2], p_full[2]
+    static constexpr int kNumBars = 1 + 2 * kMaxRing + 4 + 2;         // q, full[], empty[], s_full[2], p_full[2], drain[2]
     static constexpr int kTmemPtrOff = kBarOff + 8 * kNumBars;
     static constexpr int kAbortOff = kTmemPtrOff + 4;
     static constexpr int kQOff = 1024;
@@ -280,6 +280,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     auto bar_empty = [&](int i) { return bar0 + 8 * (1 + kMaxRing + i); };
     auto bar_s = [&](int b) { return bar0 + 8 * (1 + 2 * kMaxRing + b); };
     auto bar_p = [&](int b) { return bar0 + 8 * (3 + 2 * kMaxRing + b); };
+    auto bar_drain = [&](int who) { return bar0 + 8 * (5 + 2 * kMaxRing + who); };   // error path only
     volatile uint32_t *tmem_ptr = reinterpret_cast<volatile uint32_t *>(smem + L::kTmemPtrOff);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kAbortOff);
 
@@ -310,6 +311,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         // thread that watches the K/V tiles land (see the MMA issuers); with one row tile both p[] are per key tile
         // and both take it
         for (int t = 0; t < 2; ++t) { mbar_init(bar_s(t), 1); mbar_init(bar_p(t), 128 + ((kWatch && (!kTwo || t == 0)) ? 1 : 0)); }
+        for (int t = 0; t < 2; ++t) mbar_init(bar_drain(t), 1);
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
@@ -692,6 +694,16 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
             const unsigned long long t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 2000000ull) { }
         }
+        // Tensor memory is freed below.  MMAs that an issuing thread had queued before it gave up may still be
+        // running, so each issuing thread commits once more -- the commit completes when every tensor-core
+        // operation that thread issued has retired -- and waits for that (bounded: 2 ms is thousands of times
+        // the longest queue this block can hold; nothing waits on these two barriers otherwise).
+        if ((warp == kMmaWarp || warp == kMmaWarp2) && lane == 0) {
+            const uint32_t bar = bar_drain(warp - kMmaWarp);
+            tc_commit(bar);
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(bar, 0) && global_timer_ns() - t0 < 2000000ull) { }
+        }
         __syncthreads();
     }
     // Every result of this block is stored (the barrier above): count the block off for the merge stage of a fused
@@ -837,27 +849,60 @@ int launch_bounded_wait_selftest(int32_t *status, unsigned long long limit_ns, v
 int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
 {
     if (a.num_items == 0) return 0;
-    EncodeFn fn = get_encode_fn(err);
-    if (!fn) return int(cudaErrorNotSupported);
     const int G = a.num_q_heads / a.num_kv_heads;
     const int D = a.head_dim;
     // block shape: see launch_one
     const int shape = a.max_rows_per_item > kPrefixTileRows ? 2 : ((a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) ? 1 : 0);
     const int tile_keys = shape == 1 ? prefix_tile_keys<true>() : prefix_tile_keys<false>();
-    CUtensorMap mq, mk, mv;
-    {   // Q as (d, g, kv head, sample): a box of (64, G, 1, 128/G) lands as 128 rows ordered sample-major, g fastest
-        const cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(G), cuuint64_t(a.num_kv_heads), cuuint64_t(a.num_samples)};
-        const cuuint64_t strides[3] = {cuuint64_t(D) * 2, cuuint64_t(G) * D * 2, cuuint64_t(a.num_q_heads) * D * 2};
-        const cuuint32_t box[4] = {64, cuuint32_t(G), 1, cuuint32_t(kPrefixTileRows / G)};
-        if (!encode(fn, &mq, a.q, 4, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+    // The three tensor maps depend only on the buffers' addresses, the strides and a few plan constants, and a
+    // decode loop presents the same few buffers step after step: encoding them (three driver calls, 2-3 us) is
+    // done once per distinct key and kept in a small per-thread table.
+    struct MapKey {
+        const void *q, *k, *v;
+        int64_t stride_tok, stride_head, total_tokens;
+        int32_t num_samples, num_q_heads, num_kv_heads, head_dim, tile_keys, device;
+        bool operator==(const MapKey &o) const
+        {
+            return q == o.q && k == o.k && v == o.v && stride_tok == o.stride_tok && stride_head == o.stride_head &&
+                   total_tokens == o.total_tokens && num_samples == o.num_samples && num_q_heads == o.num_q_heads &&
+                   num_kv_heads == o.num_kv_heads && head_dim == o.head_dim && tile_keys == o.tile_keys && device == o.device;
+        }
+    };
+    struct MapEntry { MapKey key; CUtensorMap mq, mk, mv; bool valid; };
+    constexpr int kMapCache = 16;
+    thread_local MapEntry cache[kMapCache] = {};
+    thread_local int next_victim = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+    const MapKey key{a.q, a.k, a.v, a.stride_tok, a.stride_head, a.total_tokens, a.num_samples, a.num_q_heads, a.num_kv_heads,
+                     a.head_dim, tile_keys, dev};
+    MapEntry *hit = nullptr;
+    for (int i = 0; i < kMapCache && !hit; ++i)
+        if (cache[i].valid && cache[i].key == key) hit = &cache[i];
+    if (!hit) {
+        EncodeFn fn = get_encode_fn(err);
+        if (!fn) return int(cudaErrorNotSupported);
+        MapEntry e{};
+        e.key = key;
+        {   // Q as (d, g, kv head, sample): a box of (64, G, 1, 128/G) lands as 128 rows ordered sample-major, g fastest
+            const cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(G), cuuint64_t(a.num_kv_heads), cuuint64_t(a.num_samples)};
+            const cuuint64_t strides[3] = {cuuint64_t(D) * 2, cuuint64_t(G) * D * 2, cuuint64_t(a.num_q_heads) * D * 2};
+            const cuuint32_t box[4] = {64, cuuint32_t(G), 1, cuuint32_t(kPrefixTileRows / G)};
+            if (!encode(fn, &e.mq, a.q, 4, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+        }
+        {   // K and V as (d, kv head, token): a box of (64, 1, tile_keys) is one 64-wide half of a key tile
+            const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(a.num_kv_heads), cuuint64_t(a.total_tokens)};
+            const cuuint64_t strides[2] = {cuuint64_t(a.stride_head) * 2, cuuint64_t(a.stride_tok) * 2};
+            const cuuint32_t box[3] = {64, 1, cuuint32_t(tile_keys)};
+            if (!encode(fn, &e.mk, a.k, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+            if (!encode(fn, &e.mv, a.v, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
+        }
+        e.valid = true;
+        hit = &cache[next_victim];
+        next_victim = (next_victim + 1) % kMapCache;
+        *hit = e;
     }
-    {   // K and V as (d, kv head, token): a box of (64, 1, tile_keys) is one 64-wide half of a key tile
-        const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(a.num_kv_heads), cuuint64_t(a.total_tokens)};
-        const cuuint64_t strides[2] = {cuuint64_t(a.stride_head) * 2, cuuint64_t(a.stride_tok) * 2};
-        const cuuint32_t box[3] = {64, 1, cuuint32_t(tile_keys)};
-        if (!encode(fn, &mk, a.k, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
-        if (!encode(fn, &mv, a.v, 3, dims, strides, box, err)) return int(cudaErrorInvalidValue);
-    }
+    const CUtensorMap &mq = hit->mq, &mk = hit->mk, &mv = hit->mv;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc;
     if (shape == 2) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);

@@ -33,15 +33,20 @@ def stratify(success_rates: Sequence[float], m: int) -> list[int]:
 
     Experiences are sorted by ascending success rate and cut into m runs of as equal size as possible; the success
     rates at the cuts become boundary VALUES, and every experience is then re-binned by value, so that equal success
-    rates always share a level (a level may end up empty)."""
+    rates always share a level (a level may end up empty).
+
+    "As evenly as possible" is read as: run sizes differ by at most one and the n mod m larger runs come FIRST (the
+    hardest levels), the convention of numpy.array_split; the paper does not say which runs take the remainder."""
     n = len(success_rates)
     if m < 1:
         raise ValueError("need m >= 1")
     if n == 0:
         return []
     order = sorted(success_rates)
-    boundaries = [order[min(n - 1, (k * n + m - 1) // m)] for k in range(1, m)]   # first element of run k
-    return [sum(1 for b in boundaries if r >= b) for r in success_rates]
+    q, r = divmod(n, m)
+    starts = [k * q + min(k, r) for k in range(1, m)]          # index of the first element of run k
+    boundaries = [order[min(n - 1, st)] for st in starts]
+    return [sum(1 for b in boundaries if x >= b) for x in success_rates]
 
 
 def demonstrations(levels: Sequence[int], j: int) -> list[int]:

@@ -39,24 +39,13 @@ def test_named_config_every_element(name, out_dtype):
 
 
 @pytest.mark.parametrize("name", ["cfg4", "cfg5"])
-def test_full_size_config_sampled_rows(name):
-    """Full size, the launch configuration the benchmark times; the oracle computes a sample of the
-    rows one by one: rows of the shortest and longest suffixes plus 192 random rows.  Everything
-    else is checked for being finite and bounded by the value range."""
+def test_full_size_config_every_element(name):
+    """Full size, the launch configuration the benchmark times (default plan, bf16 output), every element against
+    the oracle (a few seconds of CPU time each)."""
     w = wl.make_workload(wl.CONFIGS[name], poison=True)
-    Hq = w["num_q_heads"]
-    S = w["suffix_lens"]
-    rng = np.random.default_rng(123)
-    pick = set(rng.choice(len(S) * Hq, 192, replace=False).tolist())
-    for s in (int(np.argmin(S)), int(np.argmax(S))):
-        pick.update(range(s * Hq, (s + 1) * Hq))
-    rows = np.array(sorted(pick), dtype=np.int64)
     out, lse, plan = run_gpu(w, "bf16")
-    ref_o, ref_l, _ = oracle.attend(w, rows=rows)
-    assert_close(out[rows], lse[rows], ref_o, ref_l, name)
-    assert np.isfinite(out).all() and np.isfinite(lse).all()
-    vmax = float(np.max(np.abs(wl.bf16_bits_to_f32(w["prefix_v"][:4096]))))
-    assert np.max(np.abs(out)) <= max(vmax, 6.0)        # a convex combination of N(0,1) values
+    ref_o, ref_l, _ = oracle.attend(w)
+    assert_close(out, lse, ref_o, ref_l, name)
 
 
 # ------------------------------------------------------------------ shapes around every tile / page edge

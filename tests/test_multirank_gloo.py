@@ -104,3 +104,31 @@ def test_partition_is_contiguous_complete_and_balanced():
         cost = [L[a:b].sum() + S[a * 16:b * 16].sum() for a, b in parts]
         if world <= 3:
             assert max(cost) <= 1.6 * sum(cost) / world
+
+
+def test_rank_launcher_starts_the_ranks_bench_asks_for(tmp_path):
+    """`bench.py --gpus 2`, started as a plain python process, must run as two ranks and report n_gpus 2: the decision
+    (`needs_launcher`) and the launcher itself, with a small gloo program standing in for the GPU step."""
+    import json
+    import subprocess
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2502_02534_b200.launch import rank_environment, spawn_ranks
+    assert bench.needs_launcher(2, {}) and bench.needs_launcher(8, {"PATH": "/bin"})
+    assert not bench.needs_launcher(1, {}) and not bench.needs_launcher(2, {"WORLD_SIZE": "2"})
+    env = rank_environment(1, 2, 29512, {"KEEP": "1"})
+    assert env["RANK"] == "1" and env["LOCAL_RANK"] == "1" and env["WORLD_SIZE"] == "2" and env["MASTER_ADDR"] == "127.0.0.1"
+    assert env["MASTER_PORT"] == "29512" and env["KEEP"] == "1"
+    child = os.path.join(ROOT, "tests", "rank_child.py")
+    out_path = tmp_path / "rank0.out"
+    with open(out_path, "w") as f:
+        rc = spawn_ranks(2, [sys.executable, child, "--gpus", "2"], stdout=f, timeout_s=120)
+    assert rc == 0
+    lines = [ln for ln in open(out_path).read().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                       # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["sum"] == 3.0 and line["max_ms"] == 11.0 and line["argv"] == ["--gpus", "2"]
+    # a rank that fails ends the run with its exit code, and the other rank does not linger
+    rc = spawn_ranks(2, [sys.executable, "-c", "import os, sys, time; sys.exit(7) if os.environ['RANK'] == '1' else time.sleep(60)"],
+                     timeout_s=30)
+    assert rc == 7

@@ -50,3 +50,27 @@ def test_stratification_levels():
                     assert lv[a] <= lv[b]
     lv = stratify([0.9, 0.1, 0.5], 3)
     assert demonstrations(lv, 0) == [1] and demonstrations(lv, 1) == [1, 2] and demonstrations(lv, 2) == [0, 1, 2]
+
+
+def test_stratification_cut_positions_when_n_is_not_a_multiple_of_m():
+    """Which runs take the remainder ("as evenly as possible" leaves it open; the reading is: the first n mod m runs,
+    numpy.array_split's convention).  Hand-written levels of the sorted experiences, then numpy's own split."""
+    import numpy as np
+    distinct = lambda n: [i / 100 for i in range(n)]             # already ascending, all different
+    assert ref.stratify_literal(distinct(7), 3) == [0, 0, 0, 1, 1, 2, 2] == stratify(distinct(7), 3)
+    assert ref.stratify_literal(distinct(5), 4) == [0, 0, 1, 2, 3] == stratify(distinct(5), 4)
+    assert ref.stratify_literal(distinct(6), 4) == [0, 0, 1, 1, 2, 3] == stratify(distinct(6), 4)   # ceil(k n / m) cuts would give [0,0,1,2,2,3]
+    assert ref.stratify_literal(distinct(2), 4) == [0, 3] == stratify(distinct(2), 4)   # more levels than experiences: empty runs start at the end
+    rng = random.Random(7)
+    for _ in range(300):
+        n, m = rng.randint(1, 40), rng.randint(1, 7)
+        rates = rng.sample(range(1000), n)                        # distinct, shuffled
+        expect = [0] * n
+        order = sorted(range(n), key=lambda i: rates[i])
+        for level, part in enumerate(np.array_split(np.array(order), m)):
+            for i in part:
+                expect[int(i)] = level
+        if n >= m:        # with distinct rates and no empty run, re-binning by value changes nothing
+            assert ref.stratify_literal(rates, m) == expect == stratify(rates, m)
+        else:
+            assert ref.stratify_literal(rates, m) == stratify(rates, m)
