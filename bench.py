@@ -323,6 +323,24 @@ class Runner:
             stage_ms[name] = statistics.median(ts) / per_graph
         self.plan.check_status()
         res["stage_ms"] = stage_ms
+        # the prefix stage planned for itself: the same prompts and samples with no suffix work, so that the planner
+        # cuts the items for a grid that owns the machine (in the fused step it shares the SMs with the suffix stage)
+        w = self.w
+        alone = self.psa.Plan(w["prefix_lens"], w["n_samples"], np.zeros_like(np.asarray(w["suffix_lens"])), num_q_heads=self.Hq,
+                              num_kv_heads=w["num_kv_heads"], head_dim=self.D, page_size=w["page_size"], sm_scale=w["sm_scale"],
+                              out_dtype="bf16")
+        alone.bind_workspace()
+        if alone.info.num_prefix_items:
+            fused_plan, self.plan = self.plan, alone
+            try:
+                g = self.capture(lambda i: self.step(i, "prefix"), per_graph)
+                g.replay()
+                ts = self.timed_blocks(g.replay, per_graph, min(min_ms, 30.0), 100)
+                alone.check_status()
+            finally:
+                self.plan = fused_plan
+            res["prefix_alone"] = {"ms": statistics.median(ts) / per_graph, "items": alone.info.num_prefix_items,
+                                   "tiles_per_item": alone.info.prefix_tiles_per_item}
         return res
 
     def e2e(self, budget_s=8.0):
@@ -395,6 +413,14 @@ class Runner:
             share = min(1.0, blocks / n_sms)
             kernels["prefix"].update({"blocks": blocks, "sms": n_sms, "tensor_frac_on_sms_used_of_measured":
                                       flops["prefix"] / (tf_sus * 1e12 * share) / (res["stage_ms"]["prefix"] * 1e-3)})
+        if res.get("prefix_alone"):
+            pa = res["prefix_alone"]
+            kernels["prefix_planned_alone"] = {"ms": pa["ms"], "items": pa["items"], "tiles_per_item": pa["tiles_per_item"],
+                                               "frac_of_measured": kernels["prefix"]["t_roof_ms"] / pa["ms"],
+                                               "frac_of_nominal": kernels["prefix"]["t_roof_nominal_ms"] / pa["ms"],
+                                               "achieved_tflops": flops["prefix"] / (pa["ms"] * 1e-3) / 1e12,
+                                               "achieved_gbs": bytes_["prefix"] / (pa["ms"] * 1e-3) / 1e9,
+                                               "note": "prefix stage of a plan without suffix work: the grid owns the SMs"}
         tot_b, tot_f = bytes_["prefix"] + bytes_["suffix"], flops["prefix"] + flops["suffix"]
         t_step = max(tot_b / (hbm * 1e9), tot_f / (tf_sus * 1e12)) * 1e3
         t_step_nom = max(tot_b / (NOMINAL["hbm_gbs"] * 1e9), tot_f / (NOMINAL["bf16_tflops"] * 1e12)) * 1e3
@@ -484,7 +510,7 @@ def run_psa(args, cfg):
                              "sample_tokens_per_s": value, "stage_us": {n: k[n]["ms"] * 1e3 for n in k},
                              "frac_of_measured": {**{n: k[n]["frac_of_measured"] for n in k}, "step": s["frac_of_measured"]},
                              "frac_of_nominal": {**{n: k[n]["frac_of_nominal"] for n in k}, "step": s["frac_of_nominal"]},
-                             "bound": {n: k[n]["bound"] for n in k}, "traffic": r["traffic"],
+                             "bound": {n: k[n]["bound"] for n in ("prefix", "suffix", "merge")}, "traffic": r["traffic"],
                              "plan": line["plan"], "cpu_baseline": line["cpu_baseline"]}
                 continue
             c = wl.CONFIGS[name]
@@ -496,7 +522,7 @@ def run_psa(args, cfg):
                          "stage_us": {n: k[n]["ms"] * 1e3 for n in k},
                          "frac_of_measured": {**{n: k[n]["frac_of_measured"] for n in k}, "step": s["frac_of_measured"]},
                          "frac_of_nominal": {**{n: k[n]["frac_of_nominal"] for n in k}, "step": s["frac_of_nominal"]},
-                         "bound": {n: k[n]["bound"] for n in k},
+                         "bound": {n: k[n]["bound"] for n in ("prefix", "suffix", "merge")},
                          "traffic": ncu_traffic(name, "suffix_kernel", k["suffix"]["algorithmic_bytes"]),
                          "plan": {"prefix_items": rn.info.num_prefix_items, "suffix_items": rn.info.num_suffix_items,
                                   "prefix_tiles_per_item": rn.info.prefix_tiles_per_item,

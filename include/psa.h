@@ -71,8 +71,20 @@ typedef struct {
     int32_t suffix_chunk_tokens;   /* tokens per suffix work item: 0 = planner's choice, else a multiple of 64 */
     int32_t prefix_tiles_per_item; /* 128-key tiles per prefix work item: 0 = planner's choice */
     int32_t prefix_rows_per_item;  /* query rows per prefix work item: 0 = planner's choice, else 128 or 256 */
-    int32_t reserved;   /* must be 0 */
+    int32_t prefix_kernel;         /* which prefix block shape to launch: PSA_PREFIX_KERNEL_AUTO (0) = planner's choice */
 } psa_config_t;
+
+/* Prefix block shapes (psa_config_t.prefix_kernel); a tuning knob like the three above, results are the same.
+ * Items of more than 128 query rows always take a two-row-tile shape (DECOUPLED unless COUPLED is asked for); the
+ * others apply to items of at most 128 rows. */
+enum {
+    PSA_PREFIX_KERNEL_AUTO = 0,
+    PSA_PREFIX_KERNEL_SMALL = 1,     /* one row tile, 64-key tiles, small enough to share its SM with a suffix block */
+    PSA_PREFIX_KERNEL_LONG = 2,      /* one row tile, 128-key tiles, deep ring: long HBM-bound items of few rows */
+    PSA_PREFIX_KERNEL_DECOUPLED = 3, /* two softmax warpgroups fed two score tiles ahead (on alternate key tiles when
+                                        there is one row tile) */
+    PSA_PREFIX_KERNEL_COUPLED = 4    /* two row tiles, one score buffer each (the earlier shape, kept for comparison) */
+};
 
 /* What the planner decided; for tests, logs and roofline accounting. */
 typedef struct {
@@ -284,14 +296,36 @@ psa_status_t psa_validate_page_table(const psa_plan_t *plan, const int32_t *page
  * grows by one token per decode step, up to 1024: appendix "Experiment details").  For every sample s, the rows
  * new_k[s], new_v[s] ([B, Hkv, D] bf16 device, contiguous) are written to position S_s = suffix_lens[s] of the
  * sample's page list and suffix_lens[s] becomes S_s + 1 (device memory, in place), all on `cuda_stream`.
- * The page for position S_s must already be in the sample's page list, and S_s must be below the bound the plan
- * was made with; otherwise that sample is left untouched and the status word reports PSA_ERR_BOUNDS
+ * The page for position S_s must already be in the sample's page list (a negative id there counts as missing), and
+ * S_s must be below the bound the plan was made with; otherwise that sample is left untouched and the status word reports PSA_ERR_BOUNDS
  * (psa_check_status).  The plan itself does not change: psa_decode may follow immediately.
  */
 psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void *new_v,
                            void *suffix_k_pool, void *suffix_v_pool, const int64_t pool_strides[3],
                            const int32_t *page_indptr, const int32_t *page_indices, int32_t *suffix_lens,
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * psa_append_kv with page allocation on the device.  A sample whose length S_s is a multiple of 16 needs a fresh page for
+ * its next token; here the library takes it from a caller-owned stack of free page ids instead of expecting the caller to
+ * have put it into the page list beforehand, so that a decode loop (attend, draw, append, ...) can run without the host
+ * looking at the lengths -- for instance as one replayed CUDA graph.
+ *   page_indptr   [B+1] int32 device: sample s owns the SLOTS page_indices[page_indptr[s] .. page_indptr[s+1]) (its capacity).
+ *   page_indices  int32 device, in/out: slots 0 .. ceil(S_s / 16) - 1 of a sample hold its pages; every slot beyond must
+ *                 hold a negative value until this function assigns a page to it.
+ *   free_pages    int32 device: free_pages[0 .. *free_count) are ids of pages nobody owns (a stack, top at the end).
+ *   free_count    int32 device, in/out.
+ * Samples are served in sample order, so the result does not depend on scheduling: the r-th sample (in that order) that
+ * needs a page gets free_pages[*free_count - 1 - r]; *free_count drops by the number of pages handed out.  When the stack
+ * runs out, the remaining samples that need a page are left untouched (length, pools and list unchanged) and the status
+ * word reports PSA_ERR_BOUNDS; the same holds for a sample at its planned bound or without a free slot in its list.
+ * Everything else is psa_append_kv.  Enqueues two kernels on `cuda_stream`.
+ */
+psa_status_t psa_append_kv_alloc(const psa_plan_t *plan, const void *new_k, const void *new_v,
+                                 void *suffix_k_pool, void *suffix_v_pool, const int64_t pool_strides[3],
+                                 const int32_t *page_indptr, int32_t *page_indices, int32_t *suffix_lens,
+                                 const int32_t *free_pages, int32_t *free_count,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * The step after the path, second half: draw the next token of every sample from its logits.  The paper samples its
@@ -316,6 +350,15 @@ size_t psa_sample_scratch_bytes(int32_t num_rows);
 psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
                                const float *temperature, const uint64_t *seeds, uint32_t step, int32_t *tokens,
                                void *scratch, size_t scratch_bytes, void *cuda_stream);
+/*
+ * psa_sample_tokens with the decode step kept in DEVICE memory: the kernels read *step_device where psa_sample_tokens
+ * takes `step`, and add `advance` to it once every row has been drawn.  A CUDA graph that holds this call can so be
+ * replayed step after step and still draw fresh, reproducible numbers (the paper's samples run for up to 1024 steps:
+ * appendix "Experiment details").  step_device: 4-byte aligned device pointer, in/out.  Everything else as above.
+ */
+psa_status_t psa_sample_tokens_at(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
+                                  const float *temperature, const uint64_t *seeds, uint32_t *step_device, uint32_t advance,
+                                  int32_t *tokens, void *scratch, size_t scratch_bytes, void *cuda_stream);
 
 /*
  * The paper's three "attn" tasks (appendix "Benchmark details"): softmax(S) V folded over a stream of keys in the

@@ -174,6 +174,44 @@ def append_kv(w: dict, new_k: np.ndarray, new_v: np.ndarray) -> dict:
     return out
 
 
+def append_kv_alloc(w: dict, new_k: np.ndarray, new_v: np.ndarray, free_pages, free_count: int):
+    """append_kv with pages taken from a stack, sample by sample in order.  `page_indptr` gives every sample its SLOTS
+    (capacity); a slot without a page holds a negative id; `free_pages[:free_count]` are ids nobody owns, the top of the
+    stack at the end.  A sample whose length is a multiple of the page size pops one id for its next slot; a sample that
+    cannot be served -- stack empty, no slot left, or already at `suffix_bounds[s]` when the workload carries bounds -- is
+    skipped.  Returns (new workload, new free_count, list of skipped samples); the input is left alone."""
+    page = int(w["page_size"])
+    out = dict(w)
+    out["pool_k"] = np.array(w["pool_k"], copy=True)
+    out["pool_v"] = np.array(w["pool_v"], copy=True)
+    out["page_indices"] = np.array(w["page_indices"], dtype=np.int32, copy=True)
+    lens = np.array(w["suffix_lens"], dtype=np.int32, copy=True)
+    bounds = w.get("suffix_bounds")
+    free = [int(x) for x in np.asarray(free_pages)[:free_count]]
+    skipped = []
+    for s in range(len(lens)):
+        S = int(lens[s])
+        first, cap = int(w["page_indptr"][s]), int(w["page_indptr"][s + 1]) - int(w["page_indptr"][s])
+        slot = S // page
+        if (bounds is not None and S >= int(bounds[s])) or slot >= cap:
+            skipped.append(s)
+            continue
+        if S % page == 0:                      # the token opens a new page
+            if not free:
+                skipped.append(s)
+                continue
+            out["page_indices"][first + slot] = free.pop()
+        pg = int(out["page_indices"][first + slot])
+        if pg < 0:
+            skipped.append(s)
+            continue
+        out["pool_k"][pg, :, S % page, :] = new_k[s]
+        out["pool_v"][pg, :, S % page, :] = new_v[s]
+        lens[s] = S + 1
+    out["suffix_lens"] = lens
+    return out, len(free), skipped
+
+
 def causal_attend(q, k, v, prompt_lens, sm_scale, rows=None, n_threads: int = 0):
     """Prefill: causal self-attention of packed prompts.  q [T, Hq, D], k / v [T, Hkv, D] as bf16 bits (uint16).
     Returns (out [n_rows, D], lse [n_rows]) in float64; rows = token * Hq + head."""

@@ -5,5 +5,5 @@ Every step of the path runs in the CUDA library.  There is no fallback: if
 requested, the call raises.
 """
 from .binding import (  # noqa: F401
-    PsaError, Plan, PlanInfo, decode, decode_host, decode_static, static_check_status, static_selftest_bounded_wait, append_kv, prefill, sample_tokens, attn_task, library, library_path, status_string, EXPORTED_SYMBOLS,
+    PsaError, Plan, PlanInfo, decode, decode_host, decode_static, static_check_status, static_selftest_bounded_wait, append_kv, append_kv_alloc, prefill, sample_tokens, sample_tokens_at, attn_task, library, library_path, status_string, EXPORTED_SYMBOLS,
 )

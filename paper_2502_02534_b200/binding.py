@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "psa_plan_create", "psa_plan_create_cascade", "psa_plan_create_prefill", "psa_prefill", "psa_plan_destroy", "psa_plan_get_info", "psa_plan_workspace_bytes",
     "psa_plan_bind_workspace", "psa_plan_prefix_items", "psa_plan_suffix_items",
     "psa_decode", "psa_decode_static", "psa_static_check_status", "psa_static_selftest_bounded_wait", "psa_decode_prefix", "psa_decode_suffix", "psa_decode_merge",
-    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens", "psa_attn_task",
+    "psa_decode_host_staging_bytes", "psa_decode_host", "psa_check_status", "psa_selftest_bounded_wait", "psa_append_kv", "psa_append_kv_alloc", "psa_validate_page_table", "psa_sample_scratch_bytes", "psa_sample_tokens", "psa_sample_tokens_at", "psa_attn_task",
     "psa_status_string", "psa_last_error_message", "psa_version",
 ]
 
@@ -32,7 +32,7 @@ class PsaError(RuntimeError):
 class _Config(ctypes.Structure):
     _fields_ = [("num_q_heads", c_int32), ("num_kv_heads", c_int32), ("head_dim", c_int32), ("page_size", c_int32),
                 ("sm_scale", c_float), ("out_dtype", c_int32), ("num_sms", c_int32), ("suffix_chunk_tokens", c_int32),
-                ("prefix_tiles_per_item", c_int32), ("prefix_rows_per_item", c_int32), ("reserved", c_int32)]
+                ("prefix_tiles_per_item", c_int32), ("prefix_rows_per_item", c_int32), ("prefix_kernel", c_int32)]
 
 
 class _Info(ctypes.Structure):
@@ -108,6 +108,10 @@ def library():
         lib.psa_check_status.argtypes = [P, P, P]
         lib.psa_append_kv.restype = c_int32
         lib.psa_append_kv.argtypes = [P, P, P, P, P, POINTER(c_int64), P, P, P, P, c_size_t, P]
+        lib.psa_append_kv_alloc.restype = c_int32
+        lib.psa_append_kv_alloc.argtypes = [P, P, P, P, P, POINTER(c_int64), P, P, P, P, P, P, c_size_t, P]
+        lib.psa_sample_tokens_at.restype = c_int32
+        lib.psa_sample_tokens_at.argtypes = [P, c_int32, c_int64, c_int32, c_int32, P, P, P, ctypes.c_uint32, P, P, c_size_t, P]
         lib.psa_validate_page_table.restype = c_int32
         lib.psa_validate_page_table.argtypes = [P, P, P, P, c_int64, P, c_size_t, P]
         lib.psa_sample_scratch_bytes.restype = c_size_t
@@ -162,7 +166,7 @@ class Plan:
 
     def __init__(self, prefix_lens, n_samples_per_prefix, suffix_lens, *, num_q_heads, num_kv_heads, head_dim,
                  page_size=16, sm_scale=None, out_dtype="bf16", num_sms=0, suffix_chunk_tokens=0, prefix_tiles_per_item=0,
-                 prefix_rows_per_item=0, groups=None, prefill_prompt_lens=None):
+                 prefix_rows_per_item=0, prefix_kernel=0, groups=None, prefill_prompt_lens=None):
         """``groups`` = (first_sample[], n_samples[], token_len[]) plans a cascade of shared prefixes
         (psa_plan_create_cascade); ``prefix_lens`` / ``n_samples_per_prefix`` are then ignored."""
         lib = library()
@@ -171,7 +175,7 @@ class Plan:
         self.sm_scale = float(sm_scale if sm_scale is not None else head_dim ** -0.5)
         self.out_dtype = {"bf16": PSA_OUT_BF16, "f32": PSA_OUT_F32}[out_dtype]
         cfg = _Config(num_q_heads, num_kv_heads, head_dim, page_size, self.sm_scale, self.out_dtype, num_sms,
-                      suffix_chunk_tokens, prefix_tiles_per_item, prefix_rows_per_item, 0)
+                      suffix_chunk_tokens, prefix_tiles_per_item, prefix_rows_per_item, int(prefix_kernel))
         handle = c_void_p()
         self._h = None
         if prefill_prompt_lens is not None:     # causal self-attention of whole prompts (psa_plan_create_prefill)
@@ -190,7 +194,10 @@ class Plan:
 
     def __del__(self):
         if getattr(self, "_h", None):
-            library().psa_plan_destroy(self._h)
+            try:
+                library().psa_plan_destroy(self._h)
+            except Exception:       # interpreter shutdown: the module globals are already gone
+                pass
             self._h = None
 
     @property
@@ -323,6 +330,36 @@ def append_kv(plan: Plan, new_k, new_v, suffix_k_pool, suffix_v_pool, page_indpt
     _check(library().psa_append_kv(plan.handle, _ptr(new_k), _ptr(new_v), _ptr(suffix_k_pool), _ptr(suffix_v_pool), qst,
                                    _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens), _ptr(plan.workspace),
                                    plan.workspace.numel(), _stream_ptr(stream)))
+
+
+def append_kv_alloc(plan: Plan, new_k, new_v, suffix_k_pool, suffix_v_pool, page_indptr, page_indices, suffix_lens,
+                    free_pages, free_count, *, pool_strides=None, stream=None):
+    """psa_append_kv_alloc: like append_kv, but a sample that starts a new page takes it from the stack
+    free_pages[0 .. free_count) (int32 device tensors; free_count has one element and is updated in place)."""
+    if plan.workspace is None:
+        plan.bind_workspace(stream=stream)
+    qst = _strides(pool_strides or default_pool_strides(plan), 3)
+    _check(library().psa_append_kv_alloc(plan.handle, _ptr(new_k), _ptr(new_v), _ptr(suffix_k_pool), _ptr(suffix_v_pool), qst,
+                                         _ptr(page_indptr), _ptr(page_indices), _ptr(suffix_lens), _ptr(free_pages),
+                                         _ptr(free_count), _ptr(plan.workspace), plan.workspace.numel(), _stream_ptr(stream)))
+
+
+def sample_tokens_at(logits, temperature, seeds, step_device, advance=1, tokens=None, scratch=None, *, stream=None):
+    """psa_sample_tokens_at: the decode step is read from (and advanced in) the one-element int32 device tensor
+    `step_device`, so that a captured graph holding this call can be replayed step after step."""
+    import torch
+    lib = library()
+    B, V = logits.shape
+    dtype = {torch.bfloat16: PSA_OUT_BF16, torch.float32: PSA_OUT_F32}[logits.dtype]
+    if logits.stride(1) != 1:
+        raise ValueError("logits must be contiguous along the vocabulary")
+    if tokens is None:
+        tokens = torch.empty(B, dtype=torch.int32, device=logits.device)
+    if scratch is None:
+        scratch = torch.empty(max(8, int(lib.psa_sample_scratch_bytes(B))), dtype=torch.uint8, device=logits.device)
+    _check(lib.psa_sample_tokens_at(_ptr(logits), dtype, logits.stride(0), B, V, _ptr(temperature), _ptr(seeds), _ptr(step_device),
+                                    int(advance), _ptr(tokens), _ptr(scratch), scratch.numel(), _stream_ptr(stream)))
+    return tokens
 
 
 def sample_tokens(logits, temperature, seeds, step, tokens=None, scratch=None, *, stream=None):

@@ -226,6 +226,8 @@ static psa_status_t prefix_impl(const psa_plan_t *plan, const void *q, const voi
     a.items = c.prefix_items; a.num_items = int32_t(plan->prefix_items.size());
     a.max_rows_per_item = plan->prefix_max_rows_per_item; a.max_tiles_per_item = plan->prefix_tiles_per_item;
     a.causal = plan->causal;
+    a.kernel_choice = plan->cfg.prefix_kernel;
+    a.no_suffix_stage = plan->suffix_items.empty();
     a.partial_o = c.partial_o; a.partial_lse = c.partial_lse; a.status = c.status;
     a.launch_counter = count_blocks ? c.status + psa::kPrefixLaunchWord : nullptr;
     a.done_counter = count_blocks ? c.status + psa::kPrefixDoneWord : nullptr;
@@ -445,10 +447,34 @@ psa_status_t psa_check_status(const psa_plan_t *plan, void *workspace, void *cud
     return PSA_OK;
 }
 
+static psa_status_t append_impl(const psa_plan_t *plan, const void *new_k, const void *new_v, void *suffix_k_pool,
+                                void *suffix_v_pool, const int64_t pool_strides[3], const int32_t *page_indptr,
+                                const int32_t *page_indices, int32_t *suffix_lens, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream, const int32_t *free_pages, int32_t *free_count, int32_t *page_indices_rw);
+
 psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void *new_v, void *suffix_k_pool,
                            void *suffix_v_pool, const int64_t pool_strides[3], const int32_t *page_indptr,
                            const int32_t *page_indices, int32_t *suffix_lens, void *workspace, size_t workspace_bytes,
                            void *cuda_stream)
+{
+    return append_impl(plan, new_k, new_v, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens,
+                       workspace, workspace_bytes, cuda_stream, nullptr, nullptr, nullptr);
+}
+
+psa_status_t psa_append_kv_alloc(const psa_plan_t *plan, const void *new_k, const void *new_v, void *suffix_k_pool,
+                                 void *suffix_v_pool, const int64_t pool_strides[3], const int32_t *page_indptr,
+                                 int32_t *page_indices, int32_t *suffix_lens, const int32_t *free_pages, int32_t *free_count,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!free_pages || !free_count) return fail(PSA_ERR_INVALID_ARG, "null free_pages / free_count");
+    return append_impl(plan, new_k, new_v, suffix_k_pool, suffix_v_pool, pool_strides, page_indptr, page_indices, suffix_lens,
+                       workspace, workspace_bytes, cuda_stream, free_pages, free_count, page_indices);
+}
+
+static psa_status_t append_impl(const psa_plan_t *plan, const void *new_k, const void *new_v, void *suffix_k_pool,
+                                void *suffix_v_pool, const int64_t pool_strides[3], const int32_t *page_indptr,
+                                const int32_t *page_indices, int32_t *suffix_lens, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream, const int32_t *free_pages, int32_t *free_count, int32_t *page_indices_rw)
 {
     Carved c;
     psa_status_t st = carve(plan, workspace, workspace_bytes, &c);
@@ -467,6 +493,7 @@ psa_status_t psa_append_kv(const psa_plan_t *plan, const void *new_k, const void
     a.sample_info = c.sample_info;
     a.num_samples = plan->num_samples; a.num_kv_heads = plan->cfg.num_kv_heads; a.head_dim = plan->cfg.head_dim;
     a.status = c.status;
+    a.free_pages = free_pages; a.free_count = free_count; a.page_indices_rw = page_indices_rw;
     const int rc = psa::launch_append(a, cuda_stream);
     if (rc != 0) return cuda_fail(cudaError_t(rc), "append launch");
     return PSA_OK;

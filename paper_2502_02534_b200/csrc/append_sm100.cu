@@ -27,9 +27,11 @@ append_kernel(const uint4 *__restrict__ new_k, const uint4 *__restrict__ new_v, 
     if (threadIdx.x == 0) {
         const int S = suffix_lens[s];
         const int first = page_indptr[s], n_pages = page_indptr[s + 1] - first;
-        const bool ok = S >= 0 && S < sample_info[s].suf_len_bound && S / kPageSize < n_pages;
+        bool ok = S >= 0 && S < sample_info[s].suf_len_bound && S / kPageSize < n_pages;
+        const int page = ok ? page_indices[first + S / kPageSize] : 0;
+        ok = ok && page >= 0;   // a negative id marks a slot of the list that no page has been assigned to
         sh_pos = ok ? S : -1;
-        sh_page = ok ? page_indices[first + S / kPageSize] : 0;
+        sh_page = page;
         if (!ok) atomicCAS(status, 0, int(PSA_ERR_BOUNDS));
     }
     __syncthreads();
@@ -47,6 +49,62 @@ append_kernel(const uint4 *__restrict__ new_k, const uint4 *__restrict__ new_v, 
     }
     __syncthreads();
     if (threadIdx.x == 0) suffix_lens[s] = pos + 1;
+}
+
+// Page allocation for the append: a sample whose length is a multiple of the page size needs a fresh page for its
+// next token.  One block walks the samples IN ORDER (so that the assignment does not depend on scheduling): the r-th
+// sample that needs a page takes free_pages[*free_count - 1 - r], the top of the caller's stack of free page ids, and
+// the id goes into the sample's page list at slot S / 16.  When the stack runs out the remaining samples get nothing:
+// their slot keeps its negative id, the append kernel then leaves them untouched and reports PSA_ERR_BOUNDS.
+// A sample at its planned bound, or whose list has no slot left, asks for nothing (the append kernel reports it).
+__global__ void __launch_bounds__(1024)
+allocate_pages_kernel(const int32_t *__restrict__ page_indptr, int32_t *__restrict__ page_indices,
+                      const int32_t *__restrict__ suffix_lens, const SampleInfo *__restrict__ sample_info, int num_samples,
+                      const int32_t *__restrict__ free_pages, int32_t *__restrict__ free_count, int *__restrict__ status)
+{
+    __shared__ int warp_sums[32];
+    __shared__ int base, available;
+    if (threadIdx.x == 0) { base = 0; available = max(0, *free_count); }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int s0 = 0; s0 < num_samples; s0 += blockDim.x) {
+        const int s = s0 + threadIdx.x;
+        int need = 0, slot = 0, first = 0;
+        if (s < num_samples) {
+            const int S = suffix_lens[s];
+            first = page_indptr[s];
+            slot = S / kPageSize;
+            need = S >= 0 && S < sample_info[s].suf_len_bound && S % kPageSize == 0 && slot < page_indptr[s + 1] - first;
+        }
+        // rank of this sample among the samples of the chunk that need a page (block-wide exclusive scan)
+        int incl = need;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int w = lane < int(blockDim.x >> 5) ? warp_sums[lane] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += v;
+            }
+            warp_sums[lane] = w;   // inclusive sums over warps
+        }
+        __syncthreads();
+        const int rank = base + (warp ? warp_sums[warp - 1] : 0) + incl - need;
+        if (need) {
+            if (rank < available) page_indices[first + slot] = free_pages[available - 1 - rank];
+            else atomicCAS(status, 0, int(PSA_ERR_BOUNDS));   // the stack is empty: the slot stays unassigned
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) base += warp_sums[(blockDim.x >> 5) - 1];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *free_count = available - min(available, base);
 }
 
 // Debug aid: check a page table against the plan before trusting it to the suffix stage.  One thread per sample:
@@ -83,6 +141,12 @@ int launch_validate(const int32_t *page_indptr, const int32_t *page_indices, con
 int launch_append(const AppendArgs &a, void *stream)
 {
     if (a.num_samples == 0) return 0;
+    if (a.free_pages != nullptr) {
+        allocate_pages_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+            a.page_indptr, a.page_indices_rw, a.suffix_lens, a.sample_info, a.num_samples, a.free_pages, a.free_count, a.status);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return int(e);
+    }
     append_kernel<<<a.num_samples, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4 *>(a.new_k), static_cast<const uint4 *>(a.new_v), static_cast<uint4 *>(a.pool_k),
         static_cast<uint4 *>(a.pool_v), a.stride_page, a.stride_head, a.stride_tok, a.page_indptr, a.page_indices,

@@ -122,7 +122,7 @@ psa_status_t build_plan(const psa_config_t &cfg, int32_t P, const int32_t *first
         return fail(PSA_ERR_INVALID_ARG, "sm_scale must be positive and finite");
     if (cfg.out_dtype != PSA_OUT_BF16 && cfg.out_dtype != PSA_OUT_F32)
         return fail(PSA_ERR_UNSUPPORTED, "out_dtype must be PSA_OUT_BF16 or PSA_OUT_F32");
-    if (cfg.reserved != 0) return fail(PSA_ERR_INVALID_ARG, "reserved must be 0");
+    if (cfg.prefix_kernel < 0 || cfg.prefix_kernel > PSA_PREFIX_KERNEL_COUPLED) return fail(PSA_ERR_INVALID_ARG, "prefix_kernel out of range");
     if (cfg.suffix_chunk_tokens < 0 || cfg.suffix_chunk_tokens % 64 != 0)
         return fail(PSA_ERR_INVALID_ARG, "suffix_chunk_tokens must be 0 or a multiple of 64");
     if (cfg.prefix_tiles_per_item < 0) return fail(PSA_ERR_INVALID_ARG, "prefix_tiles_per_item must be >= 0");

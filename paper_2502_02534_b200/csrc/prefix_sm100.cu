@@ -58,6 +58,10 @@ namespace psa {
 namespace {
 
 constexpr float kRescaleThreshold = 8.f; // log2 units
+// bf16 by truncation, unbiased: exponentiate x + log2(1 + 2^-9), truncate, and divide the row sum by (1 + 2^-9) at the end
+constexpr float kTruncBias = 0.0028150156f;      // log2(1 + 2^-9)
+constexpr float kTruncUnbias = 0.99805068f;      // 1 / (1 + 2^-9)
+constexpr float kTileSumLimit = 64.f * 256.f * 1.01f;   // 64 exponentials of at most 2^8 (times the factor above)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -135,22 +139,39 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A * B with A from shared memory (mma_ss_w) or from tensor memory (mma_ts_w), B from shared memory.
-// Shared-memory descriptors are given as (low word, high word): the one thread that issues every
-// MMA of a block keeps the high words (layout constants) in registers and derives each low word (the address) with
-// a single add, so that issuing stays far cheaper than the MMA itself.
-__device__ __forceinline__ void mma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                         uint32_t accumulate)
+// One lane of a converged warp.  Code guarded by this (rather than by a test of the lane index) is known to the
+// compiler to run on a single lane, so descriptors and addresses stay in the uniform datapath the tensor-core
+// instructions take their operands from; guarded by `lane == 0` every tcgen05.mma cost the issuing thread 90-130
+// cycles of register shuffling, more than the 64 cycles the instruction needs to execute.
+__device__ __forceinline__ bool elect_one()
 {
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
-__device__ __forceinline__ void mma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t accumulate)
+// D[tmem] (+)= A * B with A from shared memory (mma_ss) or from tensor memory (mma_ts), B from shared memory.
+// Shared-memory descriptors are 64-bit values: the high word holds layout constants, the low word the address
+// (in 16-byte units), so stepping through a tile is one add.  kAcc: accumulate onto D (compile-time: the predicate
+// operand is then an immediate); mma_ts_p takes the flag at run time.
+template <bool kAcc>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc)
 {
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 db, {%2, %3};\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (kAcc)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t db, uint32_t idesc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(db), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void mma_ts_p(uint32_t d_tmem, uint32_t a_tmem, uint64_t db, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns: thread = lane (row), register i = column i
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
@@ -183,17 +204,29 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// 2^x without the special-function unit: x = n + f with n the nearest integer (magic-number rounding) and f in
+// [-0.5, 0.5], a minimax cubic for 2^f (relative error below 7.5e-5, mean error 5e-6), and n added to the exponent bits.
+// Three adds, three FMAs, a maximum and two integer operations: more instructions than one ex2, but on pipes that are
+// idle while the special-function unit, one exponential per score, is the scarce resource of the softmax pass.
+__device__ __forceinline__ float poly_exp2(float x)
+{
+    x = fmaxf(x, -126.f);                        // below that the result is zero for every purpose here
+    const float t = x + 12582912.f;              // 1.5 * 2^23: n lands in the low mantissa bits
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(f, 0.0551716648f, 0.2426111251f);
+    p = fmaf(p, f, 0.6932609677f);
+    p = fmaf(p, f, 0.9999280572f);
+    // at the clamp (masked keys arrive as -inf) the value is a denormal just below 2^-126: a flushing multiply by one
+    // turns it into the exact zero that ex2 returns there
+    float r;
+    asm("mul.ftz.f32 %0, %1, 0f3F800000;" : "=f"(r) : "f"(__uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23))));
+    return r;
+}
 __device__ __forceinline__ float fast_exp2(float x)
 {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
 }
 
 // ---------------------------------------------------------------- descriptors
@@ -318,7 +351,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_ptr)), L::kTmemCols);
         tmem_relinquish();
     }
-    if (warp == kProducerWarp && lane == 0) { prefetch_tensormap(pmap_q); prefetch_tensormap(pmap_k); prefetch_tensormap(pmap_v); }
+    if (warp == kProducerWarp && elect_one()) { prefetch_tensormap(pmap_q); prefetch_tensormap(pmap_k); prefetch_tensormap(pmap_v); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -334,7 +367,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (elect_one()) {
             mbar_expect_tx(bar_q(), n_rt * L::kQTileBytes);
             for (int t = 0; t < n_rt; ++t)
                 for (int h = 0; h < L::kHalves; ++h)
@@ -358,27 +391,33 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         // issuers the waits of one overlap the MMAs of the other.
         //   two row tiles: thread 0 issues everything, thread 1 only watches the K/V tiles land (see there)
         //   one row tile:  issuer 0 issues every QK^T, issuer 1 every PV
-        if (lane == 0) {
+        if (elect_one()) {
             const int who = warp - kMmaWarp;
             auto wait_entry = [&](int e) { return mbar_wait(bar_full(e % ring), (e / ring) & 1, abort_flag); };
-            constexpr uint32_t kHiK = smem_desc_hi(1024), kHiV = smem_desc_hi(1024);
-            const uint32_t q_lo = smem_desc_lo(sbase + L::kQOff, 16);
-            const uint32_t ring_k_lo = smem_desc_lo(sbase + L::kRingOff, 16);            // K tiles: K-major, no leading offset
-            const uint32_t ring_v_lo = smem_desc_lo(sbase + L::kRingOff, L::kHalfBytes); // V tiles: MN-major, halves kHalfBytes apart
+            constexpr uint64_t kHi = uint64_t(smem_desc_hi(1024)) << 32;
+            const uint64_t q_desc = kHi | smem_desc_lo(sbase + L::kQOff, 16);
+            const uint64_t ring_k_desc = kHi | smem_desc_lo(sbase + L::kRingOff, 16);            // K tiles: K-major, no leading offset
+            const uint64_t ring_v_desc = kHi | smem_desc_lo(sbase + L::kRingOff, L::kHalfBytes); // V tiles: MN-major, halves kHalfBytes apart
             auto issue_qk = [&](int t, int sb, int kslot) {   // S[sb] = Q_t K^T, K in ring slot `kslot`
-                const uint32_t a_lo = q_lo + uint32_t(t) * (L::kQTileBytes >> 4);
-                const uint32_t b_lo = ring_k_lo + uint32_t(kslot) * (L::kTileBytes >> 4);
+                const uint64_t a = q_desc + uint32_t(t) * (L::kQTileBytes >> 4);
+                const uint64_t b = ring_k_desc + uint32_t(kslot) * (L::kTileBytes >> 4);
                 const uint32_t d = tmem_base + kColS + uint32_t(sb) * 128;
 #pragma unroll
-                for (int k = 0; k < kKSteps; ++k)
-                    mma_ss_w(d, a_lo + (((k / 4) * L::kQHalfBytes + (k % 4) * 32) >> 4), kHiK,
-                             b_lo + (((k / 4) * L::kHalfBytes + (k % 4) * 32) >> 4), kHiK, kIdescQK, k > 0);
+                for (int k = 0; k < kKSteps; ++k) {
+                    const uint64_t ak = a + (((k / 4) * L::kQHalfBytes + (k % 4) * 32) >> 4);
+                    const uint64_t bk = b + (((k / 4) * L::kHalfBytes + (k % 4) * 32) >> 4);
+                    if (k == 0) mma_ss<false>(d, ak, bk, kIdescQK);
+                    else mma_ss<true>(d, ak, bk, kIdescQK);
+                }
             };
             auto issue_pv = [&](int t, uint32_t p_tmem, int vslot, bool first) {   // O_t += P V, V in ring slot `vslot`
-                const uint32_t b_lo = ring_v_lo + uint32_t(vslot) * (L::kTileBytes >> 4);
+                const uint64_t b = ring_v_desc + uint32_t(vslot) * (L::kTileBytes >> 4);
+                const uint32_t d = tmem_base + kColO + t * D;
 #pragma unroll
-                for (int k = 0; k < kPSteps; ++k)
-                    mma_ts_w(tmem_base + kColO + t * D, p_tmem + k * 8, b_lo + ((k * 2048) >> 4), kHiV, kIdescPV, (!first || k > 0));
+                for (int k = 0; k < kPSteps; ++k) {
+                    if (k == 0) mma_ts_p(d, p_tmem, b, kIdescPV, first ? 0u : 1u);
+                    else mma_ts(d, p_tmem + k * 8, b + ((k * 2048) >> 4), kIdescPV);
+                }
             };
             auto next_slot = [&](int sl, int by) { sl += by; return sl >= ring ? sl - ring : sl; };
             if constexpr (kTwo) {
@@ -460,7 +499,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
     } else if (!kTwo && kWatch && warp == kWatchWarp) {
         // ------------------------------------------------------------ watcher (one row tile): per key tile j it waits
         // for V_j and K_{j+2} to land and then adds its arrival to p[j & 1], so that the two issuers poll one barrier each
-        if (lane == 0) {
+        if (elect_one()) {
             bool landed = true;
             for (int j = 0; landed && j < n_tiles; ++j) {
                 if (j >= 2) landed = mbar_wait(bar_p(j & 1), sphase(j - 2), abort_flag);   // one arrival per phase
@@ -513,7 +552,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 return true;
             };
 
-            float ps[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial row sums
+            float tile_sum = 0.f;   // the row's sum over this tile (times 1 + 2^-9, see exp_in_place)
             if constexpr (kTwo) {
                 // ---- S in registers; P (bf16) is written back over the first 64 columns of S.
                 // Common case: ONE pass that exponentiates against the current reference maximum while tracking the
@@ -532,30 +571,30 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                                 if (c * 32 + i >= valid) sreg[c][i] = 0xff800000u;
                     }
                 };
-                auto exp_in_place = [&](float &xmax) {   // sreg: 128 scores -> 64 words of packed bf16 P (in sreg[0], sreg[1])
-                    const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // a row that has seen no key yet: exponentiate against 0
-                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                    ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
+                // sreg: 128 scores -> 64 words of packed bf16 P (in sreg[0], sreg[1]); returns the row's sum of the tile.
+                // bf16 by truncation (a byte permute on the integer pipe: the special-function unit does the
+                // exponentials and nothing else), unbiased by exponentiating x + log2(1 + 2^-9); no running maximum: a
+                // tile sum above kKeys * 2^8 is what tells that some exponent exceeded the threshold.
+                auto exp_in_place = [&]() -> float {
+                    const float off = kTruncBias - (m_ref == -INFINITY ? 0.f : m_ref);   // no key seen yet: exponentiate against 0
+                    float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const float x0 = fmaf(__uint_as_float(sreg[c][i]), scale_log2, -m_use);
-                            const float x1 = fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, -m_use);
-                            mx[(i >> 1) & 3] = fmaxf(mx[(i >> 1) & 3], fmaxf(x0, x1));
-                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                            ps[(i >> 1) & 3] += p0 + p1;
-                            sreg[c / 2][(c % 2) * 16 + i / 2] = pack_bf16(p0, p1);
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][i]), scale_log2, off));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][i + 1]), scale_log2, off));
+                            sum[(i >> 1) & 3] += p0 + p1;
+                            sreg[c / 2][(c % 2) * 16 + i / 2] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
                         }
                     }
-                    xmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 };
                 load_s();
                 bool redo = j == 0;   // nothing to exponentiate against yet
                 if (j > 0) {
-                    float xmax;
-                    exp_in_place(xmax);
-                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold || (m_ref == -INFINITY && xmax != -INFINITY));
+                    tile_sum = exp_in_place();
+                    redo = __any_sync(0xffffffffu, !(tile_sum <= float(kKeys) * 256.f * 1.01f) || (m_ref == -INFINITY && valid > 0));
                     if (redo) load_s();
                 }
                 if (redo) {
@@ -570,8 +609,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     if (__any_sync(0xffffffffu, need)) {
                         if (!(ok = move_reference(need, tmax))) break;
                     }
-                    float xmax;
-                    exp_in_place(xmax);
+                    tile_sum = exp_in_place();
                 }
                 tmem_st32(s_addr, sreg[0]);
                 tmem_st32(s_addr + 32, sreg[1]);
@@ -583,11 +621,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                 const uint32_t p_addr = tmem_base + lane_addr + kColP + b * 64;
                 // P[b] was last read by the PV of tile j-2, which a different thread issues than the QK^T that made this S
                 if (j >= 2 && !(ok = mbar_wait(bar_empty((2 * j - 3) % ring), ((2 * j - 3) / ring) & 1, abort_flag))) break;
-                auto exp_pass = [&](float &xmax) {
-                    const float m_use = m_ref == -INFINITY ? 0.f : m_ref;   // no key seen yet: exponentiate against 0
+                auto exp_pass = [&]() -> float {   // the same truncating, bias-cancelling form as above, 32 columns at a time
+                    const float off = kTruncBias - (m_ref == -INFINITY ? 0.f : m_ref);   // no key seen yet: exponentiate against 0
                     uint32_t r[2][32];
-                    float mx[2] = {-INFINITY, -INFINITY};
-                    ps[0] = ps[1] = ps[2] = ps[3] = 0.f;
+                    float sum[4] = {0.f, 0.f, 0.f, 0.f};
                     tmem_ld32(s_addr, r[0]);
                     tmem_wait_ld();
 #pragma unroll
@@ -596,29 +633,26 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, -m_use);
-                            float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, -m_use);
+                            float x0 = fmaf(__uint_as_float(r[c & 1][i]), scale_log2, off);
+                            float x1 = fmaf(__uint_as_float(r[c & 1][i + 1]), scale_log2, off);
                             if (valid < kKeys) {   // masked keys of a ragged last tile
                                 if (c * 32 + i >= valid) x0 = -INFINITY;
                                 if (c * 32 + i + 1 >= valid) x1 = -INFINITY;
                             }
-                            mx[0] = fmaxf(mx[0], x0);
-                            mx[1] = fmaxf(mx[1], x1);
                             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                            ps[(i >> 1) & 3] += p0 + p1;
-                            pk[i / 2] = pack_bf16(p0, p1);
+                            sum[(i >> 1) & 3] += p0 + p1;
+                            pk[i / 2] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
                         }
                         tmem_st16(p_addr + c * 16, pk);
                         tmem_wait_ld();
                     }
-                    xmax = fmaxf(mx[0], mx[1]);
+                    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 };
                 bool redo = j == 0;   // nothing to exponentiate against yet
                 if (j > 0) {
-                    float xmax;
-                    exp_pass(xmax);
-                    // also redo when a row meets its first visible key (its reference maximum is still -inf)
-                    redo = __any_sync(0xffffffffu, xmax > kRescaleThreshold || (m_ref == -INFINITY && xmax != -INFINITY));
+                    tile_sum = exp_pass();
+                    // redo when an exponent exceeded the threshold (the sum tells) or a row meets its first visible key
+                    redo = __any_sync(0xffffffffu, !(tile_sum <= float(kKeys) * 256.f * 1.01f) || (m_ref == -INFINITY && valid > 0));
                 }
                 if (redo) {
                     // the tile's maximum, then the classic update, then the exponentials again
@@ -637,11 +671,10 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
                     const float tmax = scale_log2 * fmaxf(mx[0], mx[1]);
                     const bool need = tmax > m_ref + kRescaleThreshold;
                     if (!(ok = move_reference(need, tmax))) break;
-                    float xmax;
-                    exp_pass(xmax);
+                    tile_sum = exp_pass();
                 }
             }
-            l_sum += (ps[0] + ps[1]) + (ps[2] + ps[3]);
+            l_sum += tile_sum;
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p(b));
@@ -650,6 +683,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         // ring is idle by now) so that every global store instruction writes one full 4*D-byte row.
         // The release of the last V buffer follows the last MMA of the block (of both row tiles): O is final
         // and nothing reads the ring any more, so the staging tile may overlay it.
+        l_sum *= kTruncUnbias;   // the row sums carry the factor (1 + 2^-9) of the truncation trick
         if (ok) ok = mbar_wait(bar_empty((2 * n_tiles - 1) % ring), ((2 * n_tiles - 1) / ring) & 1, abort_flag);
         float *stage = reinterpret_cast<float *>(smem + L::kRingOff + t * L::kStageBytes);
         if (ok) {
@@ -698,7 +732,7 @@ prefix_body(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensor
         // running, so each issuing thread commits once more -- the commit completes when every tensor-core
         // operation that thread issued has retired -- and waits for that (bounded: 2 ms is thousands of times
         // the longest queue this block can hold; nothing waits on these two barriers otherwise).
-        if ((warp == kMmaWarp || warp == kMmaWarp2) && lane == 0) {
+        if ((warp == kMmaWarp || warp == kMmaWarp2) && elect_one()) {   // the lane that issued the MMAs
             const uint32_t bar = bar_drain(warp - kMmaWarp);
             tc_commit(bar);
             const unsigned long long t0 = global_timer_ns();
@@ -750,6 +784,439 @@ prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_c
 {
     prefix_body<D, false, false>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status, launch_counter,
                             done_counter);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Decoupled block: two softmax warpgroups ("streams") whose score tiles are produced TWO steps ahead.
+//
+// The blocks above make a stream's next score tile only after its current probabilities have been consumed (P is
+// written over S and there is one S buffer per stream), so every key tile costs a stream the whole chain
+// S ready -> softmax pass -> P ready -> PV -> QK^T -> S ready, and the tensor pipe idles for the part of it that the
+// other stream's work does not cover.  Here a key tile has 64 keys, which leaves tensor memory for TWO S buffers per
+// stream (4 x 64 columns) beside the two accumulators (2 x D columns): QK^T of step j + 2 is issued right behind PV
+// of step j, so that S of step j + 1 is already complete when a warpgroup finishes step j.  The warpgroups then run
+// their passes back to back and the issuing thread finds P waiting: the block is bound by the tensor pipe (8 SS MMAs
+// of 48 cycles + 4 TS MMAs of 64 cycles per 128 rows x 64 keys) instead of by the chain.
+//
+// Two forms of "stream":
+//   kPing == false  two ROW tiles of 128 rows share every K/V tile (items of up to 256 rows): stream t = row tile t.
+//   kPing == true   ONE row tile (items of up to 128 rows), the streams take alternate KEY tiles (stream t: tiles
+//                   t, t + 2, ...), each with its own accumulator and running (m, l); the two are combined in the
+//                   epilogue (the same identity the merge stage uses).  Both warpgroups work for every row count.
+// K and V tiles travel through a ring each; the producer issues K `kLead` tiles ahead of V (the distance between a
+// tile's QK^T and its PV).  11 warps: 0-3 / 4-7 softmax warpgroups, 8 TMA producer, 9 / 10 MMA issuer of stream 0 / 1
+// (warp 9 owns the tensor memory allocation).  The block owns its SM (193 KB of shared memory).
+template <int D, bool kPing>
+struct PrefixSmem2 {
+    static constexpr int kKeys = 64;
+    static constexpr int kHalves = D / 64;
+    static constexpr int kQTiles = kPing ? 1 : 2;
+    static constexpr int kQHalfBytes = kPrefixTileRows * 128;
+    static constexpr int kQTileBytes = kHalves * kQHalfBytes;
+    static constexpr int kHalfBytes = kKeys * 128;                    // one TMA box of K or V: 64 rows x 64 bf16
+    static constexpr int kTileBytes = kHalves * kHalfBytes;
+    static constexpr int kRK = kPing ? 7 : 6, kRV = kPing ? 5 : 4;    // ring lengths: all of the 227 KB, a tile takes 1.5-2 us to arrive
+    static constexpr int kLead = kPing ? 4 : 2;                       // K tiles issued before the first V tile
+    // barriers (8 bytes each)
+    static constexpr int kBarQ = 0, kBarKFull = 1, kBarKEmpty = kBarKFull + kRK, kBarVFull = kBarKEmpty + kRK,
+                         kBarVEmpty = kBarVFull + kRV, kBarS = kBarVEmpty + kRV, kBarP = kBarS + 4, kBarPV = kBarP + 4,
+                         kBarDone = kBarPV + 4, kBarDrain = kBarDone + 1, kNumBars = kBarDrain + 2;
+    static constexpr int kTmemPtrOff = 8 * kNumBars;
+    static constexpr int kAbortOff = kTmemPtrOff + 4;
+    static constexpr int kExchangeOff = 1024;                         // kPing: (m, l) of every row of both streams, 2 KB
+    static constexpr int kQOff = 3072;
+    static constexpr int kKRingOff = kQOff + kQTiles * kQTileBytes;
+    static constexpr int kVRingOff = kKRingOff + kRK * kTileBytes;
+    static constexpr int kTotal = kVRingOff + kRV * kTileBytes;
+    static constexpr int kStageRowFloats = D + 4;
+    static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;   // staging tile(s) overlay Q and the rings
+    static constexpr int kTmemCols = 512;                             // S[t][b] at 64 (2 t + b); O[t] at 256 + t D
+    static_assert(kAbortOff + 4 <= kExchangeOff && kTotal <= 227 * 1024 && kQTiles * kStageBytes <= kTotal - kQOff, "shared memory plan");
+};
+
+template <int D, bool kPing>
+__device__ __forceinline__ void
+prefix_body2(const CUtensorMap *pmap_q, const CUtensorMap *pmap_k, const CUtensorMap *pmap_v,
+             const PrefixItem *__restrict__ items, int group, int causal, float scale_log2,
+             float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status, int *launch_counter,
+             int *done_counter)
+{
+    using L = PrefixSmem2<D, kPing>;
+    constexpr int kKeys = L::kKeys;
+    constexpr int kProducerWarp = 8, kMmaWarp = 9;
+    constexpr int kKSteps = D / 16, kPSteps = kKeys / 16;
+    constexpr uint32_t kIdescQK = make_idesc(kKeys, false);
+    constexpr uint32_t kIdescPV = make_idesc(D, true);
+    constexpr uint32_t kColO = 256;
+
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {   // swizzled tiles need a 1024-byte aligned base; refuse to run rather than read garbage
+        if (threadIdx.x == 0) atomicCAS(status, 0, int(PSA_ERR_BOUNDS));
+        return;
+    }
+    auto bar = [&](int i) { return sbase + 8 * i; };
+    auto bar_s = [&](int t, int b) { return bar(L::kBarS + 2 * t + b); };     // S[t][b] complete (tcgen05.commit)
+    auto bar_p = [&](int t, int b) { return bar(L::kBarP + 2 * t + b); };     // P written over S[t][b] (128 softmax threads)
+    auto bar_pv = [&](int t, int b) { return bar(L::kBarPV + 2 * t + b); };   // the PV that read that P is complete: O[t] quiescent
+    volatile uint32_t *tmem_ptr = reinterpret_cast<volatile uint32_t *>(smem + L::kTmemPtrOff);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kAbortOff);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (launch_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0)
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(launch_counter) : "memory");
+    const int4 it0 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x));
+    const int4 it1 = __ldg(reinterpret_cast<const int4 *>(items + blockIdx.x) + 1);
+    const int first_token = it0.x, n_keys = it0.y, kv = it0.z, first_sample = it0.w;
+    const int n_rows = it1.x, prow0 = it1.y;
+    const int n_tiles = (n_keys + kKeys - 1) / kKeys;
+    const int samples_per_tile = kPrefixTileRows / group;
+    // stream t, step j  ->  key tile, and how many steps the stream has
+    const int n_streams = kPing ? (n_tiles > 1 ? 2 : 1) : (n_rows > kPrefixTileRows ? 2 : 1);
+    auto key_tile = [&](int t, int j) { return kPing ? 2 * j + t : j; };
+    auto n_steps = [&](int t) { return t >= n_streams ? 0 : (kPing ? (n_tiles - t + 1) / 2 : n_tiles); };
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(L::kBarQ), 1);
+        // a ring slot is free again when every stream that reads the tile has consumed it: both row tiles, or the
+        // one stream an alternate key tile belongs to
+        const int users = kPing ? 1 : n_streams;
+        for (int i = 0; i < L::kRK; ++i) { mbar_init(bar(L::kBarKFull + i), 1); mbar_init(bar(L::kBarKEmpty + i), users); }
+        for (int i = 0; i < L::kRV; ++i) { mbar_init(bar(L::kBarVFull + i), 1); mbar_init(bar(L::kBarVEmpty + i), users); }
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(L::kBarS + i), 1); mbar_init(bar(L::kBarP + i), 128); mbar_init(bar(L::kBarPV + i), 1); }
+        mbar_init(bar(L::kBarDone), 2);   // one arrival per issuing thread
+        mbar_init(bar(L::kBarDrain), 1);
+        mbar_init(bar(L::kBarDrain + 1), 1);
+        fence_barrier_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_ptr)), L::kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && elect_one()) { prefetch_tensormap(pmap_q); prefetch_tensormap(pmap_k); prefetch_tensormap(pmap_v); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (launch_counter != nullptr && blockIdx.x == 0 && threadIdx.x == 0) __threadfence();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            const int q_tiles = kPing ? 1 : n_streams;
+            mbar_expect_tx(bar(L::kBarQ), q_tiles * L::kQTileBytes);
+            for (int t = 0; t < q_tiles; ++t)
+                for (int h = 0; h < L::kHalves; ++h)
+                    tma_load_4d(sbase + L::kQOff + t * L::kQTileBytes + h * L::kQHalfBytes, pmap_q, bar(L::kBarQ), h * 64, 0, kv,
+                                first_sample + t * samples_per_tile);
+            bool ok = true;
+            auto load = [&](bool is_v, int i) {   // key tile i of K or V into its ring
+                const int ring = is_v ? L::kRV : L::kRK;
+                const int slot = i % ring, use = i / ring;
+                const uint32_t full = bar((is_v ? L::kBarVFull : L::kBarKFull) + slot), empty = bar((is_v ? L::kBarVEmpty : L::kBarKEmpty) + slot);
+                if (use > 0 && !(ok = mbar_wait(empty, (use - 1) & 1, abort_flag))) return;
+                mbar_expect_tx(full, L::kTileBytes);
+                const uint32_t dst = sbase + (is_v ? L::kVRingOff : L::kKRingOff) + slot * L::kTileBytes;
+                for (int h = 0; h < L::kHalves; ++h)
+                    tma_load_3d(dst + h * L::kHalfBytes, is_v ? pmap_v : pmap_k, full, h * 64, kv, first_token + i * kKeys);
+            };
+            for (int i = 0; ok && i < L::kLead && i < n_tiles; ++i) load(false, i);
+            for (int i = 0; ok && i < n_tiles; ++i) {
+                load(true, i);
+                if (ok && i + L::kLead < n_tiles) load(false, i + L::kLead);
+            }
+        }
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+        // ------------------------------------------------------------ MMA issuers: one elected lane per stream.
+        // A stream's issuer has about 640 tensor-pipe cycles of its own MMAs per step and the same again of the other
+        // stream's to do its waits and commits in; one thread serving both streams could not keep up (a satisfied
+        // barrier wait still costs it 100-200 cycles, and a step has three).
+        const int t = warp - kMmaWarp;
+        if (elect_one()) {
+            constexpr uint64_t kHi = uint64_t(smem_desc_hi(1024)) << 32;
+            const uint64_t q_desc = (kHi | smem_desc_lo(sbase + L::kQOff, 16)) + uint32_t(kPing ? 0 : t) * (L::kQTileBytes >> 4);
+            const uint64_t k_desc = kHi | smem_desc_lo(sbase + L::kKRingOff, 16);              // K-major, no leading offset
+            const uint64_t v_desc = kHi | smem_desc_lo(sbase + L::kVRingOff, L::kHalfBytes);   // MN-major, halves kHalfBytes apart
+            const uint32_t o_tmem = tmem_base + kColO + t * D;
+            auto wait_k = [&](int i) { return mbar_wait(bar(L::kBarKFull + i % L::kRK), (i / L::kRK) & 1, abort_flag); };
+            auto wait_v = [&](int i) { return mbar_wait(bar(L::kBarVFull + i % L::kRV), (i / L::kRV) & 1, abort_flag); };
+            auto issue_qk = [&](int b, int i) {   // S[t][b] = Q K_i^T
+                const uint64_t kb = k_desc + uint32_t(i % L::kRK) * (L::kTileBytes >> 4);
+                const uint32_t d = tmem_base + uint32_t(2 * t + b) * 64;
+#pragma unroll
+                for (int k = 0; k < kKSteps; ++k) {
+                    const uint64_t ak = q_desc + (((k / 4) * L::kQHalfBytes + (k % 4) * 32) >> 4);
+                    const uint64_t bk = kb + (((k / 4) * L::kHalfBytes + (k % 4) * 32) >> 4);
+                    if (k == 0) mma_ss<false>(d, ak, bk, kIdescQK);
+                    else mma_ss<true>(d, ak, bk, kIdescQK);
+                }
+                tc_commit(bar_s(t, b));
+                tc_commit(bar(L::kBarKEmpty + i % L::kRK));
+            };
+            auto issue_pv = [&](int b, int i, bool first) {   // O[t] += P V_i, P in the first 32 columns of S[t][b]
+                const uint64_t vb = v_desc + uint32_t(i % L::kRV) * (L::kTileBytes >> 4);
+                const uint32_t p_tmem = tmem_base + uint32_t(2 * t + b) * 64;
+#pragma unroll
+                for (int k = 0; k < kPSteps; ++k) {
+                    if (k == 0) mma_ts_p(o_tmem, p_tmem, vb, kIdescPV, first ? 0u : 1u);
+                    else mma_ts(o_tmem, p_tmem + k * 8, vb + ((k * 2048) >> 4), kIdescPV);
+                }
+                tc_commit(bar_pv(t, b));
+                tc_commit(bar(L::kBarVEmpty + i % L::kRV));
+            };
+            const int steps = n_steps(t);
+            bool ok = steps > 0;
+            if (ok) ok = mbar_wait(bar(L::kBarQ), 0, abort_flag);
+            // prologue: the stream's first two score tiles
+            for (int j = 0; ok && j < 2 && j < steps; ++j) {
+                const int i = key_tile(t, j);
+                if (!(ok = wait_k(i))) break;
+                tc_fence_after();
+                issue_qk(j, i);
+            }
+            for (int j = 0; ok && j < steps; ++j) {
+                const int i = key_tile(t, j), b = j & 1;
+                if (!(ok = wait_v(i))) break;
+                if (!(ok = mbar_wait(bar_p(t, b), (j >> 1) & 1, abort_flag))) break;
+                tc_fence_after();
+                issue_pv(b, i, j == 0);
+                if (j + 2 < steps) {
+                    const int i2 = key_tile(t, j + 2);
+                    if (!(ok = wait_k(i2))) break;
+                    tc_fence_after();
+                    issue_qk(b, i2);   // overwrites P of step j: ordered behind the PV just issued
+                }
+            }
+            // when this barrier flips, every MMA of both issuers is complete
+            if (ok && steps > 0) tc_commit(bar(L::kBarDone));
+            else mbar_arrive(bar(L::kBarDone));
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------ softmax warpgroups + epilogue
+        const int t = warp >> 2;                       // stream
+        const int row = (warp & 3) * 32 + lane;        // row inside the row tile = TMEM lane
+        const int row_tile = kPing ? 0 : t;
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t o_addr = tmem_base + lane_addr + kColO + t * D;
+        const int my_steps = n_steps(t);
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        uint32_t sreg[2][32];
+        for (int j = 0; j < my_steps; ++j) {
+            const int b = j & 1, i = key_tile(t, j);
+            const uint32_t s_addr = tmem_base + lane_addr + uint32_t(2 * t + b) * 64;
+            if (!(ok = mbar_wait(bar_s(t, b), (j >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            int valid = n_keys - i * kKeys;
+            if (causal) valid = min(valid, first_sample + (row_tile * kPrefixTileRows + row) / group - (first_token + i * kKeys) + 1);
+            auto load_s = [&]() {
+                tmem_ld32(s_addr, sreg[0]);
+                tmem_ld32(s_addr + 32, sreg[1]);
+                tmem_wait_ld();
+                if (valid < kKeys) {   // ragged last tile, or the diagonal of a prefill: masked keys become -inf
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c * 32 + e >= valid) sreg[c][e] = 0xff800000u;
+                }
+            };
+            // 64 scores -> 32 words of packed bf16 P in sreg[0]; returns the row's sum of this tile.
+            // The special-function unit is the scarce pipe here (one exponential per score), so nothing else may use
+            // it: bf16 comes from TRUNCATING p (a byte permute on the integer pipe) instead of a rounding conversion,
+            // and the bias of truncation (half a unit in the last place on average) is cancelled by exponentiating
+            // x + log2(1 + 2^-9): every p -- and with it the row sum, which is corrected once in the epilogue --
+            // carries the factor (1 + 2^-9).  No running maximum either: if every exponent is below the threshold the
+            // tile sum is at most 64 * 2^8, so a sum above that bound is what sends the tile to the slow path.
+            auto exp_in_place = [&]() -> float {
+                const float off = kTruncBias - (m_ref == -INFINITY ? 0.f : m_ref);   // a row that has seen no key yet: exponentiate against 0
+                float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        // every third pair takes the polynomial: with two warps per scheduler the pass is bound by the
+                        // special-function unit, and a third of the work is what the other pipes absorb for free
+                        const bool poly = ((e >> 1) % 3) == 2;
+                        const float x0 = fmaf(__uint_as_float(sreg[c][e]), scale_log2, off), x1 = fmaf(__uint_as_float(sreg[c][e + 1]), scale_log2, off);
+                        const float p0 = poly ? poly_exp2(x0) : fast_exp2(x0), p1 = poly ? poly_exp2(x1) : fast_exp2(x1);
+                        ps[(e >> 1) & 3] += p0 + p1;
+                        sreg[0][c * 16 + e / 2] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
+                    }
+                return (ps[0] + ps[1]) + (ps[2] + ps[3]);
+            };
+            auto move_reference = [&](bool need, float m_new) -> bool {
+                const float alpha = need ? fast_exp2(m_ref - m_new) : 1.f;   // 0 on the stream's first tile
+                if (j > 0) {
+                    // O[t] must be quiescent: the PV of this stream's previous step has to be complete
+                    if (!mbar_wait(bar_pv(t, (j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag)) return false;
+                    tc_fence_after();
+                    uint32_t oreg[32];
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(o_addr + c * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
+                        tmem_st32(o_addr + c * 32, oreg);
+                    }
+                    tmem_wait_st();
+                }
+                l_sum *= alpha;
+                if (need) m_ref = m_new;
+                return true;
+            };
+            load_s();
+            float tile_sum = 0.f;
+            bool redo = j == 0;   // nothing to exponentiate against yet
+            if (j > 0) {
+                // common case: ONE pass against the current reference maximum; S is still intact (P not stored yet),
+                // so a tile with an exponent above the threshold -- or a row's first visible key -- is simply done again
+                tile_sum = exp_in_place();
+                redo = __any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit) || (m_ref == -INFINITY && valid > 0));
+                if (redo) load_s();
+            }
+            if (redo) {
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sreg[c][e]));
+                const float tmax = scale_log2 * fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                const bool need = tmax > m_ref + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    if (!(ok = move_reference(need, tmax))) break;
+                }
+                tile_sum = exp_in_place();
+            }
+            tmem_st32(s_addr, sreg[0]);
+            l_sum += tile_sum;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p(t, b));
+        }
+        // ---- epilogue.  Every MMA of the block is complete (O final, Q and the rings idle): the staging tile(s) may
+        // overlay them, so that every global store instruction writes one full row.
+        l_sum *= kTruncUnbias;   // the row sums carry the factor (1 + 2^-9) of the truncation trick
+        const bool active = kPing || t < n_streams;
+        if (active) {
+            if (ok) ok = mbar_wait(bar(L::kBarDone), 0, abort_flag);
+            if (ok) tc_fence_after();
+            float *stage = reinterpret_cast<float *>(smem + L::kQOff) + (kPing ? 0 : t * (L::kStageBytes / 4));
+            float *mine = stage + row * L::kStageRowFloats;
+            if constexpr (!kPing) {
+                if (ok) {
+                    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;   // a row that saw no key in this item: O = 0, lse = -inf
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t oreg[32];
+                        tmem_ld32(o_addr + c * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4 *>(mine + c * 32 + e) =
+                                make_float4(__uint_as_float(oreg[e]) * inv, __uint_as_float(oreg[e + 1]) * inv,
+                                            __uint_as_float(oreg[e + 2]) * inv, __uint_as_float(oreg[e + 3]) * inv);
+                    }
+                    const int r = t * kPrefixTileRows + row;
+                    if (r < n_rows) partial_lse[prow0 + r] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+                }
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");   // the four warps of this row tile
+            } else {
+                // combine the two streams of a row: with M = max(m_0, m_1) and a_t = 2^(m_t - M),
+                //   l = a_0 l_0 + a_1 l_1,   out = (a_0 O_0 + a_1 O_1) / l.
+                // (m, l) cross through shared memory; stream t then finishes the column half t of every row, reading
+                // both accumulators from tensor memory (a warp reaches the same 32 lanes in either).
+                float2 *exch = reinterpret_cast<float2 *>(smem + L::kExchangeOff);
+                exch[t * kPrefixTileRows + row] = make_float2(m_ref, l_sum);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                const float2 other = exch[(1 - t) * kPrefixTileRows + row];
+                const float m0 = t == 0 ? m_ref : other.x, l0 = t == 0 ? l_sum : other.y;
+                const float m1 = t == 0 ? other.x : m_ref, l1 = t == 0 ? other.y : l_sum;
+                const float top = fmaxf(m0, m1);
+                const float a0 = m0 == -INFINITY ? 0.f : fast_exp2(m0 - top), a1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - top);
+                const float l = a0 * l0 + a1 * l1;
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const bool have1 = n_streams > 1;    // otherwise O_1 was never written
+                if (ok) {
+                    const uint32_t o0 = tmem_base + lane_addr + kColO, o1 = o0 + D;
+                    const float w0 = a0 * inv, w1 = a1 * inv;
+#pragma unroll 1
+                    for (int c = t * (D / 64); c < (t + 1) * (D / 64); ++c) {   // 32-column pieces of this stream's half
+                        uint32_t r0[32], r1[32];
+                        tmem_ld32(o0 + c * 32, r0);
+                        if (have1) tmem_ld32(o1 + c * 32, r1);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            float v[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                v[u] = __uint_as_float(r0[e + u]) * w0;
+                                if (have1) v[u] = fmaf(__uint_as_float(r1[e + u]), w1, v[u]);
+                            }
+                            *reinterpret_cast<float4 *>(mine + c * 32 + e) = make_float4(v[0], v[1], v[2], v[3]);
+                        }
+                    }
+                    if (t == 0 && row < n_rows) partial_lse[prow0 + row] = l > 0.f ? (top + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            if (!*abort_flag) {
+                constexpr int kLanesPerRow = D / 4;                    // float4 per row: 32 or 16
+                constexpr int kRowsPerInstr = 32 / kLanesPerRow;       // 1 or 2
+                const int sub = lane / kLanesPerRow, col = (lane % kLanesPerRow) * 4;
+                const int tile_row0 = kPing ? 0 : t * kPrefixTileRows;
+                const int rows_here = min(kPrefixTileRows, n_rows - tile_row0);
+                const int n_writers = kPing ? 8 : 4, writer = kPing ? warp : (warp & 3);
+                for (int r = writer * kRowsPerInstr + sub; r < rows_here; r += n_writers * kRowsPerInstr) {
+                    const float4 v = *reinterpret_cast<const float4 *>(stage + r * L::kStageRowFloats + col);
+                    *reinterpret_cast<float4 *>(partial_o + size_t(prow0 + tile_row0 + r) * D + col) = v;
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, int(PSA_ERR_TIMEOUT));
+        // let copies that were already issued land before the block's shared memory is released
+        if (warp == kProducerWarp && lane == 0) {
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 2000000ull) { }
+        }
+        // MMAs queued before the issuing thread gave up may still run: one more commit completes when all of them
+        // have retired; wait for it (bounded) before tensor memory is freed
+        if ((warp == kMmaWarp || warp == kMmaWarp + 1) && elect_one()) {
+            const uint32_t drain = bar(L::kBarDrain + warp - kMmaWarp);
+            tc_commit(drain);
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(drain, 0) && global_timer_ns() - t0 < 2000000ull) { }
+        }
+        __syncthreads();
+    }
+    if (done_counter != nullptr && threadIdx.x == 0)
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(done_counter) : "memory");
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+}
+
+template <int D, bool kPing>
+__global__ void __launch_bounds__(352, 1)
+prefix_kernel_decoupled(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_v, const PrefixItem *__restrict__ items, int group, int causal,
+                        float scale_log2, float *__restrict__ partial_o, float *__restrict__ partial_lse, int *__restrict__ status,
+                        int *launch_counter, int *done_counter)
+{
+    prefix_body2<D, kPing>(&map_q, &map_k, &map_v, items, group, causal, scale_log2, partial_o, partial_lse, status, launch_counter,
+                           done_counter);
 }
 
 // Self-test of the bounded wait: one block waits on a barrier that nothing ever arrives on.  The wait must give
@@ -838,6 +1305,31 @@ int launch_one(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk
                                   a.partial_lse, a.status, a.launch_counter, a.done_counter));
 }
 
+template <int D, bool kPing>
+int launch_decoupled(const PrefixArgs &a, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, cudaStream_t st)
+{
+    using L = PrefixSmem2<D, kPing>;
+    auto kern = prefix_kernel_decoupled<D, kPing>;
+    static PerDeviceOnce once;   // per instantiation
+    const int cfg_rc = once.ensure([&] {
+        return int(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    });
+    if (cfg_rc != 0) return cfg_rc;
+    const float scale_log2 = a.sm_scale * 1.4426950408889634f;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(a.num_items);
+    lc.blockDim = dim3(352);   // two softmax warpgroups, producer, one MMA issuer per stream
+    lc.dynamicSmemBytes = L::kTotal;
+    lc.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = 1;
+    return int(cudaLaunchKernelEx(&lc, kern, mq, mk, mv, a.items, a.num_q_heads / a.num_kv_heads, int(a.causal), scale_log2, a.partial_o,
+                                  a.partial_lse, a.status, a.launch_counter, a.done_counter));
+}
+
 }  // namespace
 
 int launch_bounded_wait_selftest(int32_t *status, unsigned long long limit_ns, void *stream)
@@ -851,9 +1343,19 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     if (a.num_items == 0) return 0;
     const int G = a.num_q_heads / a.num_kv_heads;
     const int D = a.head_dim;
-    // block shape: see launch_one
-    const int shape = a.max_rows_per_item > kPrefixTileRows ? 2 : ((a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) ? 1 : 0);
-    const int tile_keys = shape == 1 ? prefix_tile_keys<true>() : prefix_tile_keys<false>();
+    // Block shape.  0: one row tile, long (HBM-bound items of few rows); 1: one row tile, small (shares its SM with a
+    // suffix block); 2: two row tiles, coupled (kept for comparison); 3: decoupled, two row tiles; 4: decoupled, one
+    // row tile with the streams on alternate key tiles.  a.kernel_choice forces one where the rows allow it.
+    int shape;
+    if (a.max_rows_per_item > kPrefixTileRows) shape = a.kernel_choice == PSA_PREFIX_KERNEL_COUPLED ? 2 : 3;
+    else if (a.kernel_choice == PSA_PREFIX_KERNEL_SMALL) shape = 1;
+    else if (a.kernel_choice == PSA_PREFIX_KERNEL_LONG) shape = 0;
+    else if (a.kernel_choice == PSA_PREFIX_KERNEL_DECOUPLED) shape = 4;
+    // no suffix stage in this plan (a prefix-only step): nothing to share the SM with, so rows that fill most of a
+    // row tile take the decoupled block with its streams on alternate key tiles
+    else if (a.no_suffix_stage && a.max_rows_per_item > 64 && a.max_tiles_per_item >= 2) shape = 4;
+    else shape = (a.max_tiles_per_item <= 2 || a.max_rows_per_item > 64) ? 1 : 0;
+    const int tile_keys = (shape == 0 || shape == 2) ? kPrefixTileKeys : 64;
     // The three tensor maps depend only on the buffers' addresses, the strides and a few plan constants, and a
     // decode loop presents the same few buffers step after step: encoding them (three driver calls, 2-3 us) is
     // done once per distinct key and kept in a small per-thread table.
@@ -905,7 +1407,9 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     const CUtensorMap &mq = hit->mq, &mk = hit->mk, &mv = hit->mv;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc;
-    if (shape == 2) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
+    if (shape == 3) rc = D == 128 ? launch_decoupled<128, false>(a, mq, mk, mv, st) : launch_decoupled<64, false>(a, mq, mk, mv, st);
+    else if (shape == 4) rc = D == 128 ? launch_decoupled<128, true>(a, mq, mk, mv, st) : launch_decoupled<64, true>(a, mq, mk, mv, st);
+    else if (shape == 2) rc = D == 128 ? launch_one<128, 2>(a, mq, mk, mv, st) : launch_one<64, 2>(a, mq, mk, mv, st);
     else if (shape == 1) rc = D == 128 ? launch_one<128, 1>(a, mq, mk, mv, st) : launch_one<64, 1>(a, mq, mk, mv, st);
     else rc = D == 128 ? launch_one<128, 0>(a, mq, mk, mv, st) : launch_one<64, 0>(a, mq, mk, mv, st);
     if (rc != 0 && err) *err = std::string("prefix launch: ") + cudaGetErrorString(cudaError_t(rc));

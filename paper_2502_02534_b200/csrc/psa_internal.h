@@ -148,6 +148,8 @@ struct PrefixArgs {
     int32_t num_items;
     int32_t max_rows_per_item, max_tiles_per_item;  // over all items of the plan
     bool causal = false;  // prefill: row (token) i sees keys up to its own packed token index
+    int32_t kernel_choice = 0;   // PSA_PREFIX_KERNEL_*: 0 = by the shape of the items
+    bool no_suffix_stage = false;   // the plan has no suffix work at all: the prefix grid has the SMs to itself
     float *partial_o, *partial_lse;  // device
     int32_t *status;                 // device
     int32_t *launch_counter = nullptr, *done_counter = nullptr;   // device; when set: block 0 adds 1 to the first at its start,
@@ -196,6 +198,11 @@ struct AppendArgs {
     const SampleInfo *sample_info;
     int32_t num_samples, num_kv_heads, head_dim;
     int32_t *status;
+    // page allocation (all null: every page is already in the lists): a stack of free page ids and its height,
+    // and the page lists as writable memory
+    const int32_t *free_pages = nullptr;
+    int32_t *free_count = nullptr;
+    int32_t *page_indices_rw = nullptr;
 };
 int launch_append(const AppendArgs &a, void *stream);
 int launch_validate(const int32_t *page_indptr, const int32_t *page_indices, const int32_t *suffix_lens,

@@ -71,8 +71,10 @@ __device__ __forceinline__ unsigned long long make_key(float score, uint32_t ind
 template <bool kF32>
 __global__ void __launch_bounds__(kSampleThreads)
 sample_kernel(const void *__restrict__ logits, int64_t row_stride, int vocab, int splits, const float *__restrict__ temperature,
-              const unsigned long long *__restrict__ seeds, uint32_t step, unsigned long long *__restrict__ cells)
+              const unsigned long long *__restrict__ seeds, uint32_t step_value, const uint32_t *__restrict__ step_device,
+              unsigned long long *__restrict__ cells)
 {
+    const uint32_t step = step_device ? __ldg(step_device) : step_value;   // a replayed graph reads the step from memory
     const int row = blockIdx.y, split = blockIdx.x;
     const float T = __ldg(temperature + row);
     const bool greedy = !(T > 0.f);
@@ -140,10 +142,13 @@ sample_kernel(const void *__restrict__ logits, int64_t row_stride, int vocab, in
     if ((threadIdx.x & 31) == 0 && key != 0ull) atomicMax(cells + row, key);
 }
 
-__global__ void sample_finalize_kernel(const unsigned long long *__restrict__ cells, int num_rows, int32_t *__restrict__ tokens)
+__global__ void sample_finalize_kernel(const unsigned long long *__restrict__ cells, int num_rows, int32_t *__restrict__ tokens,
+                                       uint32_t *step_device, uint32_t advance)
 {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < num_rows) tokens[r] = int32_t(0xFFFFFFFFu - uint32_t(cells[r]));
+    // every block of the drawing kernel has read the step by now (this kernel follows it in the stream)
+    if (step_device != nullptr && r == 0) *step_device += advance;
 }
 
 }  // namespace
@@ -151,9 +156,9 @@ __global__ void sample_finalize_kernel(const unsigned long long *__restrict__ ce
 
 extern "C" size_t psa_sample_scratch_bytes(int32_t num_rows) { return num_rows > 0 ? size_t(num_rows) * 8 : 0; }
 
-extern "C" psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
-                                          const float *temperature, const uint64_t *seeds, uint32_t step, int32_t *tokens,
-                                          void *scratch, size_t scratch_bytes, void *cuda_stream)
+static psa_status_t sample_impl(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
+                                const float *temperature, const uint64_t *seeds, uint32_t step, uint32_t *step_device, uint32_t advance,
+                                int32_t *tokens, void *scratch, size_t scratch_bytes, void *cuda_stream)
 {
     using psa::set_last_error;
     if (num_rows < 0 || vocab < 0) return set_last_error(PSA_ERR_INVALID_ARG, "negative num_rows or vocab");
@@ -181,11 +186,29 @@ extern "C" psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dty
     auto *cells = static_cast<unsigned long long *>(scratch);
     const auto *sd = reinterpret_cast<const unsigned long long *>(seeds);
     if (logits_dtype == PSA_OUT_F32)
-        psa::sample_kernel<true><<<grid, psa::kSampleThreads, 0, st>>>(logits, row_stride, vocab, splits, temperature, sd, step, cells);
+        psa::sample_kernel<true><<<grid, psa::kSampleThreads, 0, st>>>(logits, row_stride, vocab, splits, temperature, sd, step, step_device, cells);
     else
-        psa::sample_kernel<false><<<grid, psa::kSampleThreads, 0, st>>>(logits, row_stride, vocab, splits, temperature, sd, step, cells);
-    psa::sample_finalize_kernel<<<(num_rows + 255) / 256, 256, 0, st>>>(cells, num_rows, tokens);
+        psa::sample_kernel<false><<<grid, psa::kSampleThreads, 0, st>>>(logits, row_stride, vocab, splits, temperature, sd, step, step_device, cells);
+    psa::sample_finalize_kernel<<<(num_rows + 255) / 256, 256, 0, st>>>(cells, num_rows, tokens, step_device, advance);
     e = cudaGetLastError();
     if (e != cudaSuccess) return set_last_error(PSA_ERR_CUDA, std::string("sampling launch: ") + cudaGetErrorString(e));
     return PSA_OK;
+}
+
+extern "C" psa_status_t psa_sample_tokens(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
+                                          const float *temperature, const uint64_t *seeds, uint32_t step, int32_t *tokens,
+                                          void *scratch, size_t scratch_bytes, void *cuda_stream)
+{
+    return sample_impl(logits, logits_dtype, row_stride, num_rows, vocab, temperature, seeds, step, nullptr, 0u, tokens, scratch,
+                       scratch_bytes, cuda_stream);
+}
+
+extern "C" psa_status_t psa_sample_tokens_at(const void *logits, int32_t logits_dtype, int64_t row_stride, int32_t num_rows, int32_t vocab,
+                                             const float *temperature, const uint64_t *seeds, uint32_t *step_device, uint32_t advance,
+                                             int32_t *tokens, void *scratch, size_t scratch_bytes, void *cuda_stream)
+{
+    if (!step_device || reinterpret_cast<uintptr_t>(step_device) % 4)
+        return psa::set_last_error(PSA_ERR_INVALID_ARG, "step_device must be a 4-byte aligned device pointer");
+    return sample_impl(logits, logits_dtype, row_stride, num_rows, vocab, temperature, seeds, 0u, step_device, advance, tokens, scratch,
+                       scratch_bytes, cuda_stream);
 }
