@@ -45,10 +45,13 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # with `scaled_from` were not captured themselves: traffic grows in proportion to the tokens a launch streams, and the
 # figure is the captured configuration's bytes per algorithmic byte times this configuration's algorithmic bytes.
 NCU_TRAFFIC = {
-    "cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68271539 + 18168},
+    "cfg2": {"kernel": "suffix_kernel", "bytes_per_launch": 68273408 + 56576},      # 1.0052 x the algorithmic bytes
+    "cfg3": {"kernel": "suffix_kernel", "bytes_per_launch": 264009728 + 237312},    # 1.0031 x
 }
 NCU_TRAFFIC_SOURCE = {"suffix_kernel": ("paper_2502_02534_b200/csrc/suffix_sm100.cu", "498b791d8050fd97")}
-NCU_TRAFFIC_RATIO = {}       # kernel -> measured DRAM bytes per algorithmic byte (from the captured configurations)
+# measured DRAM bytes per algorithmic byte of the largest captured configuration (cfg3); scales the configurations that
+# are too large to capture under a profiler (cfg4, cfg5: 2.2 GB per launch), whose traffic grows with the tokens streamed
+NCU_TRAFFIC_RATIO = {"suffix_kernel": (264009728 + 237312) / 263438152}
 
 
 def ncu_traffic(config_name, kernel, algorithmic_bytes):

@@ -198,7 +198,11 @@ int launch_merge(const MergeArgs &a, void *stream, std::string *err)
     const int counted_blocks = (a.prefix_counters && a.status) ? a.prefix_blocks : 0;
     cudaError_t e;
     const bool small = rows <= 4096;   // few rows: latency matters, fetch 16 partial rows at a time
-    if (a.head_dim == 128 && small)
+    const bool large = rows > 8192;    // many rows: occupancy matters more than loads in flight per warp (4 rows at a time, 2x the warps per SM)
+    if (a.head_dim == 128 && large)
+        e = cudaLaunchKernelEx(&lc, merge_kernel<128, 4>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
+                               a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse, a.prefix_counters, counted_blocks, a.status);
+    else if (a.head_dim == 128 && small)
         e = cudaLaunchKernelEx(&lc, merge_kernel<128, 16>, a.sample_info, a.suffix_lens, a.partial_o, a.partial_lse, rows,
                                a.num_q_heads, group, a.chunk_tokens, f32, a.out, a.lse, a.prefix_counters, counted_blocks, a.status);
     else if (a.head_dim == 128)

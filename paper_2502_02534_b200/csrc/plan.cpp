@@ -8,7 +8,9 @@
 // small pieces are not preferred.
 #include <algorithm>
 #include <cstring>
+#include <functional>
 #include <limits>
+#include <queue>
 
 #include "psa_internal.h"
 
@@ -56,10 +58,35 @@ int choose_prefix_tiles_per_item(const std::vector<int64_t> &tiles, const std::v
             longest = std::max(longest, len);
             partial += double(partial_rows_per_split[p] * splits) * steps_per_partial_row;
         }
-        double cost = std::max(longest, 1.1 * sum / num_sms) + partial;
+        // Blocks that own their SM (two row tiles, or a step without a suffix stage) run in waves of num_sms: the stage
+        // lasts as long as the busiest SM when the items are dealt out longest first, and 144 items of 17 steps beat
+        // 160 items of 16 (measured on 2 x 128 rows x 16384 keys x 8 heads: 21.3 against 33.6 us).
+        double stage = std::max(longest, 1.1 * sum / num_sms);
+        if (owns_sm || sm_time_weight == 0.0) {
+            std::vector<double> lens;
+            for (size_t p = 0; p < tiles.size(); ++p) {
+                if (tiles[p] == 0) continue;
+                const int64_t splits = ceil_div(tiles[p], T);
+                const int64_t per = tiles[p] / splits, extra = tiles[p] % splits;
+                for (int64_t j = 0; j < splits; ++j)
+                    lens.insert(lens.end(), size_t(groups[p]), step_weight * double(per + (j < extra ? 1 : 0)) + overhead);
+            }
+            std::sort(lens.begin(), lens.end(), std::greater<double>());
+            std::priority_queue<double, std::vector<double>, std::greater<double>> sms;   // finish time of every SM
+            for (int i = 0; i < num_sms; ++i) sms.push(0.0);
+            double makespan = 0.0;
+            for (double len : lens) {
+                const double t = sms.top() + len;
+                sms.pop();
+                sms.push(t);
+                makespan = std::max(makespan, t);
+            }
+            stage = makespan;
+        }
+        double cost = stage + partial;
         if (owns_sm && suffix_bytes > 0.0) {
             const double step_us = 1.5, hbm = 6.4e6 /* bytes per us */, per_sm = 7.2e4;
-            const double t_prefix = std::max(longest, 1.1 * sum / num_sms) * step_us;
+            const double t_prefix = stage * step_us;
             const double free_sms = std::max(0.0, double(num_sms) - items);
             const double rate = std::max(0.0, std::min(hbm - prefix_bytes / t_prefix, free_sms * per_sm));
             cost += std::max(0.0, suffix_bytes - rate * t_prefix) / hbm / step_us;
