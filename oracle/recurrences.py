@@ -59,52 +59,62 @@ def logits(w: dict, s: int, h: int):
     return float(w["sm_scale"]) * (K @ q), V
 
 
+def _running_maximum(x):
+    """M_t = max(x_0 .. x_t) and the factor exp(M_{t-1} - M_t) by which everything accumulated before step t shrinks
+    when the maximum moves (0 at t = 0: the state starts at m = -inf, l = 0, o = 0)."""
+    x = np.asarray(x, dtype=np.float64)
+    M = np.maximum.accumulate(x) if len(x) else x
+    before = np.concatenate([[-math.inf], M[:-1]]) if len(x) else x
+    with np.errstate(invalid="ignore"):
+        keep = np.where(before == -math.inf, 0.0, np.exp(before - M))
+    return M, keep
+
+
 def task0_maxsum(x, V):
-    """Task 0 ("MaxSum"): running max m, running sum l, output normalised at every step.
-    State starts at (-inf, 0, 0)."""
-    D = V.shape[1]
-    m, l, o = -math.inf, 0.0, np.zeros(D)
-    for s_t, v_t in zip(x, V):
-        m_next = max(m, s_t)
-        l_prime = math.exp(m - m_next) * l
-        p = math.exp(s_t - m_next)
-        l_next = p + l_prime
-        o = (l_prime * o + p * v_t) / l_next
-        m, l = m_next, l_next
-    return o, m, l
+    """Task 0 ("MaxSum"): one operator carries (m, l, o) with o normalised after EVERY key.  In closed form the state
+    after t keys is m_t = max_j x_j, l_t = sum_j exp(x_j - m_t), o_t = sum_j exp(x_j - m_t) v_j / l_t (j <= t); stepping
+    from t - 1 to t, l_t = l_{t-1} exp(m_{t-1} - m_t) + exp(x_t - m_t) and the normalised o moves toward v_t by the new
+    key's share of the sum, o_t = o_{t-1} + (exp(x_t - m_t) / l_t) (v_t - o_{t-1})."""
+    V = np.asarray(V, dtype=np.float64)
+    M, keep = _running_maximum(x)
+    weight = np.exp(np.asarray(x, dtype=np.float64) - M) if len(M) else M
+    l, o = 0.0, np.zeros(V.shape[1])
+    for t in range(len(M)):
+        l = l * keep[t] + weight[t]
+        o = o + (weight[t] / l) * (V[t] - o)
+    return o, (float(M[-1]) if len(M) else -math.inf), l
 
 
 def _exp_max_diff(x):
-    """Shared first stage of Tasks 1 and 2: per step emit e = exp(s - m_new) and the
-    decay d = exp(m_old - m_new) of everything accumulated so far."""
-    m = -math.inf
-    for s_t in x:
-        m_next = max(m, s_t)
-        yield math.exp(s_t - m_next), math.exp(m - m_next), m_next
-        m = m_next
+    """Stage one of Tasks 1 and 2 ("ExpMaxDiff") as a stream: for every key its weight e_t = exp(x_t - m_t) at the new
+    running maximum, the factor d_t = exp(m_{t-1} - m_t) for what came before, and m_t."""
+    M, keep = _running_maximum(x)
+    e = np.exp(np.asarray(x, dtype=np.float64) - M) if len(M) else M
+    return list(zip(e, keep, M))
 
 
 def task1_divsum(x, V):
-    """Task 1: "ExpMaxDiff" feeds "DivSum", which keeps (l, o) with o normalised each step."""
-    D = V.shape[1]
-    l, o, m = 0.0, np.zeros(D), -math.inf
+    """Task 1: "ExpMaxDiff" feeds "DivSum", which sees only (e_t, d_t, v_t): it keeps the sum l and the NORMALISED output,
+    l_t = d_t l_{t-1} + e_t,  o_t = (d_t l_{t-1} o_{t-1} + e_t v_t) / l_t  (the two-operand weighted mean of the old
+    output and the new value)."""
+    V = np.asarray(V, dtype=np.float64)
+    l, o, m = 0.0, np.zeros(V.shape[1]), -math.inf
     for (e, d, m), v_t in zip(_exp_max_diff(x), V):
-        l_prime = d * l
-        l_next = e + l_prime
-        o = (l_prime * o + e * v_t) / l_next
-        l = l_next
-    return o, m, l
+        carried = d * l
+        l = carried + e
+        o = (carried * o + e * v_t) / l
+    return o, float(m), l
 
 
 def task2_deferred(x, V):
-    """Task 2: "ExpMaxDiff" feeds two weighted sums (scalar r, vector acc) that are only
-    divided at the end -- the form every GPU attention kernel uses."""
-    D = V.shape[1]
-    r, acc, m = 0.0, np.zeros(D), -math.inf
+    """Task 2: "ExpMaxDiff" feeds two plain weighted sums, r_t = d_t r_{t-1} + e_t and acc_t = d_t acc_{t-1} + e_t v_t,
+    divided ONCE at the end: the form every fast kernel of the library uses."""
+    V = np.asarray(V, dtype=np.float64)
+    r, acc, m = 0.0, np.zeros(V.shape[1]), -math.inf
     for (e, d, m), v_t in zip(_exp_max_diff(x), V):
-        r = r * d + e
-        acc = acc * d + e * v_t
-    return acc / r, m, r
+        r = d * r + e
+        acc = d * acc + e * v_t
+    return acc / r, float(m), r
 
 
 def merge_partials(outs, lses):

@@ -42,28 +42,28 @@ __global__ void attn_task_kernel(const __nv_bfloat16 *__restrict__ q, const __nv
             if (i < per) dot = fmaf(qv[i], __bfloat162float(k[size_t(j) * head_dim + lane * per + i]), dot);
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
-        const float s_t = sm_scale * dot;
-        const float m_next = fmaxf(m, s_t);
-        const float e = expf(s_t - m_next);          // stage one of tasks 1 and 2 ("ExpMaxDiff"); p of task 0
-        const float d = expf(m - m_next);            // decay of the accumulated state; exp(-inf) = 0 on the first key
+        // One key: the running sum is brought to the new maximum and takes the key's weight, l <- l 2^... in natural
+        // units: l <- l exp(m - m') + exp(s - m').  What differs between the forms is what the output carries.
+        const float score = sm_scale * dot;
+        const float top = fmaxf(m, score);
+        const float weight = expf(score - top);
+        const float keep = expf(m - top);            // share of the old maximum's scale that survives; 0 on the first key
+        l = fmaf(l, keep, weight);
         if constexpr (kTask == 2) {
-            l = l * d + e;
+            // deferred division: the output stays un-normalised at the scale of the running maximum
 #pragma unroll
             for (int i = 0; i < kMaxPerLane; ++i)
-                if (i < per) o[i] = fmaf(e, __bfloat162float(v[size_t(j) * head_dim + lane * per + i]), o[i] * d);
+                if (i < per) o[i] = fmaf(weight, __bfloat162float(v[size_t(j) * head_dim + lane * per + i]), o[i] * keep);
         } else {
-            // tasks 0 and 1 carry the same numbers; task 0 forms l' = exp(m - m') l in one operator, task 1 gets d from
-            // the stage before -- the arithmetic per step is identical, the output is normalised here and now
-            const float l_prime = d * l;
-            const float l_next = e + l_prime;
-            const float inv = 1.f / l_next;
+            // normalised at every step (tasks 0 and 1 carry the same numbers; the paper splits the step into one
+            // operator or two): the normalised output is a running weighted mean, and a new key moves it toward its
+            // value by the key's share of the sum so far, o <- o + (weight / l) (v - o)
+            const float share = weight / l;
 #pragma unroll
             for (int i = 0; i < kMaxPerLane; ++i)
-                if (i < per)
-                    o[i] = fmaf(l_prime, o[i], e * __bfloat162float(v[size_t(j) * head_dim + lane * per + i])) * inv;
-            l = l_next;
+                if (i < per) o[i] = fmaf(share, __bfloat162float(v[size_t(j) * head_dim + lane * per + i]) - o[i], o[i]);
         }
-        m = m_next;
+        m = top;
     }
     const float fin = (kTask == 2 && l > 0.f) ? 1.f / l : 1.f;   // the one deferred division
 #pragma unroll

@@ -106,6 +106,31 @@ def test_multi_split_prefix_and_multi_chunk_suffix_small_sm_count():
         check(w, "f32", what=f"sms{sms}", num_sms=sms)
 
 
+# ------------------------------------------------------------------ every prefix block shape
+@pytest.mark.parametrize("kernel", [1, 2, 3, 4])          # small, long, decoupled, coupled (PSA_PREFIX_KERNEL_*)
+def test_every_prefix_block_shape_against_the_oracle(kernel):
+    """The planner picks a block shape by the items' rows and lengths; here each shape is forced in turn over row counts
+    and prefix lengths around its tile edges (64- and 128-key tiles, one and two row tiles, one and several key ranges
+    per prompt), every element against the oracle.  Items of more than 128 rows take a two-row-tile shape regardless."""
+    shapes = [(128, 4, 5, 333), (128, 4, 32, 64), (128, 4, 32, 65), (128, 8, 16, 1000), (64, 4, 20, 700), (64, 8, 7, 129),
+              (128, 1, 100, 4097), (128, 2, 64, 63), (128, 4, 70, 777), (128, 4, 64, 2000), (64, 2, 150, 500), (128, 4, 40, 1),
+              (128, 4, 40, 127), (128, 4, 40, 128), (128, 4, 40, 192), (128, 4, 40, 193)]
+    for D, G, N, L in shapes:
+        w = wl.make_workload(cfg(head_dim=D, num_q_heads=2 * G, num_kv_heads=2, samples_per_prefix=N, prefix_len=(L, L),
+                                 suffix_len=(0, 60)), poison=True)
+        for tiles in (0, 1, 3):
+            check(w, "f32", what=f"kernel {kernel} D{D} G{G} N{N} L{L} tiles {tiles}", prefix_kernel=kernel, prefix_tiles_per_item=tiles)
+
+
+def test_prefix_only_plan_takes_the_decoupled_block_and_matches():
+    """A step without any suffix work (every S_s = 0) lets the prefix grid own the SMs; the planner then picks the
+    decoupled block on alternate key tiles for rows that fill most of a row tile."""
+    c = cfg(samples_per_prefix=30, num_q_heads=8, num_kv_heads=2, prefix_len=(1500, 1500), suffix_len=(0, 0))
+    w = wl.make_workload(c, poison=True)
+    check(w, "f32", what="prefix only")
+    check(w, "bf16", what="prefix only bf16")
+
+
 # ------------------------------------------------------------------ layouts, plan reuse
 def test_strided_layouts_head_major_prefix_and_token_major_pool():
     import torch
