@@ -29,8 +29,11 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
     constexpr int V = D / 32;  // floats per lane: 2 or 4
     // kChunk rows are fetched together (registers: kChunk float4 per lane)
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
-    if (row >= num_rows) return;
+    // a warp past the last row repeats the last row's work and stores nothing: every warp of the block then reaches
+    // the block-wide barrier below
+    const int row_id = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
+    const bool live = row_id < num_rows;
+    const int row = live ? row_id : num_rows - 1;
     const int s = row / num_q_heads, h = row % num_q_heads;
     const int kv = h / group, g = h % group;
 
@@ -69,8 +72,8 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
     // counters wrap together).  The launch was announced before the suffix grid could start and every prefix block
     // was running before the first suffix block, so the count is complete or about to be; the wait is bounded all
     // the same.  It sits BEFORE the wait for the suffix grid, off the critical path.
+    int lag = 0;
     if (prefix_blocks > 0) {
-        int lag = 0;
         if (lane == 0) {
             unsigned long long t0 = 0;
             for (uint32_t spins = 0;; ++spins) {
@@ -90,8 +93,13 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
         }
         lag = __shfl_sync(0xffffffffu, lag, 0);
         __syncwarp();   // lane 0's acquire load orders the other lanes' reads of the partial results as well
-        if (lag > 0) return;   // timed out: the row stays unwritten, the status word says why
     }
+    // EVERY warp of the block must have read the counters before ANY warp lets the next kernel start: the block
+    // counts as having released its dependents as soon as one of its threads has, and the next step's prefix grid
+    // announces itself in the same counters the moment it is scheduled -- a warp still polling (it sleeps 200 ns
+    // between polls) would then wait for a launch that itself waits for this grid.
+    __syncthreads();
+    if (prefix_blocks > 0 && lag > 0) return;   // timed out: the row stays unwritten, the status word says why
     // launched as a programmatic dependent: the partial results exist only after the preceding grids completed
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // the next kernel in the stream (typically the next step's prefix stage) may set itself up meanwhile;
@@ -156,6 +164,7 @@ merge_kernel(const SampleInfo *__restrict__ sample_info, const int32_t *__restri
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] *= inv;
     }
+    if (!live) return;
     if (out_is_f32) {
         float *dst = static_cast<float *>(out) + size_t(row) * D + lane * V;
         if constexpr (V == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);

@@ -1350,7 +1350,10 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     if (a.max_rows_per_item > kPrefixTileRows) shape = a.kernel_choice == PSA_PREFIX_KERNEL_COUPLED ? 2 : 3;
     else if (a.kernel_choice == PSA_PREFIX_KERNEL_SMALL) shape = 1;
     else if (a.kernel_choice == PSA_PREFIX_KERNEL_LONG) shape = 0;
-    else if (a.kernel_choice == PSA_PREFIX_KERNEL_DECOUPLED) shape = 4;
+    // the decoupled block on alternate key tiles only in prefix-only steps (the case it is planned for): forced into a
+    // step that also has a suffix stage, replayed back to back from a CUDA graph with prefix items much longer than the
+    // suffix stage, it ended runs with a launch failure whose cause has not been found; there the request is not honoured
+    else if (a.kernel_choice == PSA_PREFIX_KERNEL_DECOUPLED && a.no_suffix_stage) shape = 4;
     // no suffix stage in this plan (a prefix-only step): nothing to share the SM with, so rows that fill most of a
     // row tile take the decoupled block with its streams on alternate key tiles
     else if (a.no_suffix_stage && a.max_rows_per_item > 64 && a.max_tiles_per_item >= 2) shape = 4;
