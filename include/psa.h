@@ -82,8 +82,7 @@ enum {
     PSA_PREFIX_KERNEL_SMALL = 1,     /* one row tile, 64-key tiles, small enough to share its SM with a suffix block */
     PSA_PREFIX_KERNEL_LONG = 2,      /* one row tile, 128-key tiles, deep ring: long HBM-bound items of few rows */
     PSA_PREFIX_KERNEL_DECOUPLED = 3, /* two softmax warpgroups fed two score tiles ahead (on alternate key tiles when
-                                        there is one row tile; for items of at most 128 rows honoured only in plans
-                                        without suffix work, otherwise the planner's choice stands) */
+                                        there is one row tile); the block owns its SM */
     PSA_PREFIX_KERNEL_COUPLED = 4    /* two row tiles, one score buffer each (the earlier shape, kept for comparison) */
 };
 

@@ -805,7 +805,7 @@ prefix_kernel_one_long(const __grid_constant__ CUtensorMap map_q, const __grid_c
 //                   epilogue (the same identity the merge stage uses).  Both warpgroups work for every row count.
 // K and V tiles travel through a ring each; the producer issues K `kLead` tiles ahead of V (the distance between a
 // tile's QK^T and its PV).  11 warps: 0-3 / 4-7 softmax warpgroups, 8 TMA producer, 9 / 10 MMA issuer of stream 0 / 1
-// (warp 9 owns the tensor memory allocation).  The block owns its SM (193 KB of shared memory).
+// (warp 9 owns the tensor memory allocation).  The block owns its SM (all 227 KB of shared memory at head dimension 128).
 template <int D, bool kPing>
 struct PrefixSmem2 {
     static constexpr int kKeys = 64;
@@ -815,7 +815,13 @@ struct PrefixSmem2 {
     static constexpr int kQTileBytes = kHalves * kQHalfBytes;
     static constexpr int kHalfBytes = kKeys * 128;                    // one TMA box of K or V: 64 rows x 64 bf16
     static constexpr int kTileBytes = kHalves * kHalfBytes;
-    static constexpr int kRK = kPing ? 7 : 6, kRV = kPing ? 5 : 4;    // ring lengths: all of the 227 KB, a tile takes 1.5-2 us to arrive
+    // Ring lengths: all of the 227 KB, a tile takes 1.5-2 us to arrive.  With alternate key tiles the lengths must be
+    // EVEN, so that a slot only ever holds tiles of one stream: that stream's issuer then waits on every phase of the
+    // slot's "landed" barrier in turn.  With an odd length a slot would alternate between the streams, each issuer
+    // would see only every other phase, and a parity wait two phases ahead of the barrier reads as satisfied -- the
+    // issuer would run ahead of a tile of the other stream that is still in flight (seen as a launch failure when
+    // the block shared the memory system with a bandwidth-bound grid and tiles landed far out of order).
+    static constexpr int kRK = 6, kRV = kPing ? 6 : 4;
     static constexpr int kLead = kPing ? 4 : 2;                       // K tiles issued before the first V tile
     // barriers (8 bytes each)
     static constexpr int kBarQ = 0, kBarKFull = 1, kBarKEmpty = kBarKFull + kRK, kBarVFull = kBarKEmpty + kRK,
@@ -832,6 +838,7 @@ struct PrefixSmem2 {
     static constexpr int kStageBytes = kPrefixTileRows * kStageRowFloats * 4;   // staging tile(s) overlay Q and the rings
     static constexpr int kTmemCols = 512;                             // S[t][b] at 64 (2 t + b); O[t] at 256 + t D
     static_assert(kAbortOff + 4 <= kExchangeOff && kTotal <= 227 * 1024 && kQTiles * kStageBytes <= kTotal - kQOff, "shared memory plan");
+    static_assert(!kPing || (kRK % 2 == 0 && kRV % 2 == 0), "a ring slot must belong to one stream");
 };
 
 template <int D, bool kPing>
@@ -1350,10 +1357,7 @@ int launch_prefix(const PrefixArgs &a, void *stream, std::string *err)
     if (a.max_rows_per_item > kPrefixTileRows) shape = a.kernel_choice == PSA_PREFIX_KERNEL_COUPLED ? 2 : 3;
     else if (a.kernel_choice == PSA_PREFIX_KERNEL_SMALL) shape = 1;
     else if (a.kernel_choice == PSA_PREFIX_KERNEL_LONG) shape = 0;
-    // the decoupled block on alternate key tiles only in prefix-only steps (the case it is planned for): forced into a
-    // step that also has a suffix stage, replayed back to back from a CUDA graph with prefix items much longer than the
-    // suffix stage, it ended runs with a launch failure whose cause has not been found; there the request is not honoured
-    else if (a.kernel_choice == PSA_PREFIX_KERNEL_DECOUPLED && a.no_suffix_stage) shape = 4;
+    else if (a.kernel_choice == PSA_PREFIX_KERNEL_DECOUPLED) shape = 4;
     // no suffix stage in this plan (a prefix-only step): nothing to share the SM with, so rows that fill most of a
     // row tile take the decoupled block with its streams on alternate key tiles
     else if (a.no_suffix_stage && a.max_rows_per_item > 64 && a.max_tiles_per_item >= 2) shape = 4;
