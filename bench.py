@@ -216,10 +216,17 @@ class Runner:
             self.g_lse = torch.empty((world, self.B, self.Hq), dtype=torch.float32, device="cuda")
             self.full_out = torch.empty((self.B, world * self.Hq, self.D), dtype=torch.bfloat16, device="cuda")
             self.full_lse = torch.empty((self.B, world * self.Hq), dtype=torch.float32, device="cuda")
-        self.plan = psa.Plan(w["prefix_lens"], w["n_samples"], w["suffix_lens"], num_q_heads=self.Hq,
-                             num_kv_heads=w["num_kv_heads"], head_dim=self.D, page_size=w["page_size"],
-                             sm_scale=w["sm_scale"], out_dtype="bf16")
-        self.plan.bind_workspace()
+        # planning is host work done once per batch shape, outside the decode loop: timed on its own (plan + work lists to the device)
+        plan_ms = []
+        for _ in range(5):
+            t0 = time.perf_counter()
+            self.plan = psa.Plan(w["prefix_lens"], w["n_samples"], w["suffix_lens"], num_q_heads=self.Hq,
+                                 num_kv_heads=w["num_kv_heads"], head_dim=self.D, page_size=w["page_size"],
+                                 sm_scale=w["sm_scale"], out_dtype="bf16")
+            self.plan.bind_workspace()
+            torch.cuda.synchronize()
+            plan_ms.append((time.perf_counter() - t0) * 1e3)
+        self.plan_host_ms = statistics.median(plan_ms)
         self.info = self.plan.info
         self.ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
 
@@ -312,6 +319,11 @@ class Runner:
         self.plan.check_status()
         res = {"block_ms": times, "ms_step_median": statistics.median(times) / K, "ms_step_min": min(times) / K,
                "blocks": len(times), "launch": launch}
+        if use_graph and self.n_copies > 1:
+            # side note: the same steps on ONE input copy, which then stays in L2 (not a roofline figure)
+            g_warm = self.capture(lambda i: self.step(0), per_graph)
+            g_warm.replay()
+            res["warm_l2_ms_per_step"] = statistics.median(self.timed_blocks(g_warm.replay, per_graph, min(min_ms, 20.0), 100)) / per_graph
         if with_eager:
             n = min(K, 500)
             res["eager_ms_per_step"] = statistics.median(self.timed_blocks(lambda: [self.step(i) for i in range(n)], n, 20.0, 20)) / n
@@ -497,6 +509,7 @@ def run_psa(args, cfg):
             "gpu_launches": run.info.kernel_launches * args.steps * res["blocks"],
             "e2e": e2e, "roofline": roof, "kernels": kernels, "eager_ms_per_step": res.get("eager_ms_per_step"),
             "step_roofline": step_roof, "clocks": clocks, "input_checksum": wl.checksum(run.w),
+            "plan_host_ms": run.plan_host_ms, "warm_l2_ms_per_step": res.get("warm_l2_ms_per_step"),
         }
         line["cpu_baseline"] = run.cpu_baseline(10.0) if world == 1 else None   # reported at one GPU only
     del run
@@ -514,7 +527,8 @@ def run_psa(args, cfg):
                              "frac_of_measured": {**{n: k[n]["frac_of_measured"] for n in k}, "step": s["frac_of_measured"]},
                              "frac_of_nominal": {**{n: k[n]["frac_of_nominal"] for n in k}, "step": s["frac_of_nominal"]},
                              "bound": {n: k[n]["bound"] for n in ("prefix", "suffix", "merge")}, "traffic": r["traffic"],
-                             "plan": line["plan"], "cpu_baseline": line["cpu_baseline"]}
+                             "plan": line["plan"], "cpu_baseline": line["cpu_baseline"], "plan_host_ms": line["plan_host_ms"],
+                             "warm_l2_step_us": None if line["warm_l2_ms_per_step"] is None else line["warm_l2_ms_per_step"] * 1e3}
                 continue
             c = wl.CONFIGS[name]
             rn = Runner(c, 0, 1, "prompts", max(8, min(args.steps, 200)), max(3, min(args.warmup, 10)), quiet)
@@ -530,7 +544,8 @@ def run_psa(args, cfg):
                          "plan": {"prefix_items": rn.info.num_prefix_items, "suffix_items": rn.info.num_suffix_items,
                                   "prefix_tiles_per_item": rn.info.prefix_tiles_per_item,
                                   "suffix_chunk_tokens": rn.info.suffix_chunk_tokens},
-                         "cpu_baseline": rn.cpu_baseline(5.0)}
+                         "cpu_baseline": rn.cpu_baseline(5.0), "plan_host_ms": rn.plan_host_ms,
+                         "warm_l2_step_us": None if rs.get("warm_l2_ms_per_step") is None else rs["warm_l2_ms_per_step"] * 1e3}
             del rn
             torch.cuda.empty_cache()
         line["per_config"] = per
