@@ -549,3 +549,29 @@ def test_two_plans_on_two_streams_with_their_own_workspaces():
         ref_o, ref_l, _ = oracle.attend(w)
         B, Hq, D = out.shape
         assert_close(out.double().cpu().numpy().reshape(B * Hq, D), lse.double().cpu().numpy().reshape(-1), ref_o, ref_l, "two streams")
+
+
+# ------------------------------------------------------------------ seeded draws over shapes and planner knobs
+@pytest.mark.parametrize("seed", range(24))
+def test_drawn_shapes_and_planner_knobs_against_the_oracle(seed):
+    """Shapes nobody picked by hand: prompts, samples, heads, lengths, paging and the planner's knobs (block shape, key tiles
+    and rows per item, suffix chunk, SM count) drawn from a seeded generator, every element against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    D = int(rng.choice([64, 128]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.choice([1, 2, 3]))
+    P = int(rng.choice([1, 1, 2, 5]))
+    N = int(rng.choice([1, 3, 16, 33, 64 // G + 1, 256 // G]))
+    hi = int(rng.choice([1, 70, 200, 700, 2100]))
+    lo = hi if rng.random() < 0.5 else max(1, hi // 4)
+    s_hi = int(rng.choice([0, 17, 100, 400]))
+    c = cfg(num_prefixes=P, samples_per_prefix=N, num_q_heads=G * Hkv, num_kv_heads=Hkv, head_dim=D, prefix_len=(lo, hi),
+            suffix_len=(0, s_hi), permute_pages=bool(rng.random() < 0.5), seed=500 + seed)
+    w = wl.make_workload(c, poison=True)
+    knobs = {}
+    if rng.random() < 0.7: knobs["prefix_kernel"] = int(rng.integers(0, 5))
+    if rng.random() < 0.6: knobs["prefix_tiles_per_item"] = int(rng.choice([1, 2, 3, 5]))
+    if rng.random() < 0.4: knobs["prefix_rows_per_item"] = int(rng.choice([128, 256]))
+    if rng.random() < 0.5: knobs["suffix_chunk_tokens"] = int(rng.choice([64, 128, 256]))
+    if rng.random() < 0.3: knobs["num_sms"] = int(rng.choice([1, 7, 148]))
+    check(w, str(rng.choice(["f32", "bf16"])), what=f"seed {seed}: {c} {knobs}", **knobs)
